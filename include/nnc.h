@@ -1,0 +1,188 @@
+/*
+ * nnc.h -- C ABI of the B200-native Qwen3 forward pass (libnnc.so).
+ *
+ * The paper frames LLM deployment as "prepare the model once ahead of time, then run a prompt phase followed
+ * by token-by-token decoding at batch 1, reporting decode tokens/s" (Section 4, Evaluation; Section 3.3.1 for
+ * laying constants out once where the kernels read them).  The three main calls mirror that framing:
+ *
+ *     nnc_model_create(config, weights)   one-time weight repack + workspace carve-up
+ *     nnc_prefill(tokens)                 the prompt phase
+ *     nnc_decode_step(token) -> logits    one decoding step (the HBM-bound hot path)
+ *
+ * Conventions
+ *   - Plain C, no exceptions.  Every function that can fail returns an int status: NNC_OK (0) or a negative
+ *     nnc_status.  nnc_last_error() gives a human-readable line for the last failure of that model.
+ *   - "DEVICE pointer" = CUDA global memory on the device that was current in nnc_model_create.
+ *     "HOST pointer" = ordinary host memory.  Unless a parameter says HOST it is a DEVICE pointer.
+ *   - The library never allocates or frees device memory: the caller supplies one workspace at create time
+ *     (nnc_workspace_bytes tells how large) and owns it; it must stay alive until nnc_model_destroy.
+ *   - All work is enqueued on the CUDA stream given at create time (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and is asynchronous unless a function says it synchronises.
+ *   - Errors that the host can see (bad configuration, null pointers, cache overflow, batch too large,
+ *     workspace too small) are returned before anything is launched and leave the model unchanged.  Launch
+ *     errors reported by the CUDA runtime are returned as NNC_ERR_CUDA.  Kernels never trap or assert; every
+ *     device-side wait is bounded and reports through a status word that nnc_device_status() reads.
+ *   - All matrices are bf16, row-major W[out][in] (y = W x); bf16 values are IEEE bfloat16 bit patterns.
+ *   - The sequences of a batch advance in lock step: they all hold the same number of cached positions.
+ */
+#ifndef NNC_H_
+#define NNC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NNC_OK = 0,
+    NNC_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, unsupported shape */
+    NNC_ERR_WORKSPACE = -2,     /* workspace smaller than nnc_workspace_bytes(), or misaligned */
+    NNC_ERR_CAPACITY = -3,      /* cache length + new tokens > max_seq, batch > max_batch, tokens > max_tokens */
+    NNC_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed; see nnc_last_error */
+    NNC_ERR_DEVICE_STATUS = -5  /* a kernel reported a bounded wait that ran out */
+} nnc_status;
+
+typedef struct nnc_model nnc_model; /* opaque; host struct owned by the library */
+
+/* Model and capacity description.  Supported: head_dim == 128; n_q_heads a multiple of n_kv_heads with at
+ * most 8 query heads per KV head; hidden, intermediate multiples of 64; everything positive. */
+typedef struct {
+    int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, intermediate, vocab;
+    int32_t max_seq;        /* KV-cache capacity in positions per sequence */
+    int32_t max_batch;      /* sequences held in the cache */
+    int32_t max_tokens;     /* most tokens one nnc_prefill call may carry (batch * n_tokens); >= max_batch */
+    int32_t tie_embeddings; /* 1: the lm_head is the embedding matrix */
+    float rms_eps;          /* 1e-6 for Qwen3 */
+    float rope_theta;       /* 1e6 for Qwen3 */
+} nnc_config;
+
+/* Per-layer weights: DEVICE pointers, bf16.  Read only during nnc_model_create (they are repacked into the
+ * workspace) and may be freed by the caller afterwards.
+ *   wq [n_q_heads*128][hidden]   wk, wv [n_kv_heads*128][hidden]   wo [hidden][n_q_heads*128]
+ *   w_gate, w_up [intermediate][hidden]   w_down [hidden][intermediate]
+ *   g_in, g_post [hidden] (RMSNorm gains before attention / before the MLP)   g_q, g_k [128] (per-head
+ *   query / key RMSNorm gains, shared by the heads of the layer) */
+typedef struct {
+    const void *wq, *wk, *wv, *wo, *w_gate, *w_up, *w_down;
+    const void *g_in, *g_post, *g_q, *g_k;
+} nnc_layer_weights;
+
+typedef struct {
+    const void *embed;               /* DEVICE [vocab][hidden] */
+    const void *lm_head;             /* DEVICE [vocab][hidden]; NULL when tie_embeddings */
+    const void *g_final;             /* DEVICE [hidden] */
+    const nnc_layer_weights *layers; /* HOST array of n_layers entries (holding DEVICE pointers) */
+} nnc_weights;
+
+/* Bytes of workspace nnc_model_create needs for this configuration (repacked weights, KV cache, RoPE table,
+ * activations, split-K scratch).  Returns 0 for an invalid configuration.  Pure host arithmetic. */
+size_t nnc_workspace_bytes(const nnc_config *config);
+
+/* Ahead-of-time preparation (the paper's "constants laid out once", Section 3.3.1): validates the
+ * configuration, carves the workspace (256-byte aligned DEVICE pointer, at least nnc_workspace_bytes), builds
+ * the RoPE table on the host in double precision, and repacks the weights on the device: Wq|Wk|Wv are
+ * concatenated row-wise, gate/up rows are interleaved pairwise (row 2i = gate_i, row 2i+1 = up_i) so that one
+ * warp owns both halves of a SwiGLU output.  Synchronises the stream before returning.  *out is set only on
+ * success.  The cache starts empty. */
+int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream, nnc_model **out);
+
+/* Releases the host struct, CUDA graphs and tensor maps.  Synchronises the stream.  NULL is ignored. */
+void nnc_model_destroy(nnc_model *model);
+
+/* Prompt phase (Section 4: a prompt is processed, then decoding starts).  tokens: int32 [batch][n_tokens],
+ * ids in [0, vocab); out-of-range ids are clamped on the device.  The tokens take positions len .. len +
+ * n_tokens - 1 of every sequence, their K/V are appended, and len grows by n_tokens.
+ * logits: fp32 [batch][vocab] (last position of each sequence), or [batch][n_tokens][vocab] when
+ * all_positions != 0; may be NULL to skip the lm_head. */
+int nnc_prefill(nnc_model *model, const int32_t *tokens, int32_t batch, int32_t n_tokens, float *logits,
+                int32_t all_positions);
+
+/* One decoding step (Section 4: throughput is measured over this stage).  tokens: int32 [batch]; each
+ * sequence's token takes position len; len grows by one.  logits: fp32 [batch][vocab].  argmax: int32
+ * [batch] or NULL; lowest index wins ties.  At batch 1 the whole step is one CUDA graph launch (captured on
+ * first use for the given buffers and re-used while they stay the same). */
+int nnc_decode_step(nnc_model *model, const int32_t *tokens, int32_t batch, float *logits, int32_t *argmax);
+
+/* End-to-end variants with HOST buffers: copy the tokens to the device, run the step, copy logits (and the
+ * argmax, if not NULL) back, and synchronise the stream before returning.  HOST pointers throughout; pinned
+ * memory makes the copies faster but is not required.  logits_host may be NULL when only argmax is wanted. */
+int nnc_decode_step_host(nnc_model *model, const int32_t *tokens_host, int32_t batch, float *logits_host,
+                         int32_t *argmax_host);
+int nnc_prefill_host(nnc_model *model, const int32_t *tokens_host, int32_t batch, int32_t n_tokens,
+                     float *logits_host, int32_t all_positions);
+
+/* Set the raw cache contents of one layer of one sequence, positions [0, n_pos): k, v DEVICE bf16
+ * [n_kv_heads][n_pos][128] (K as the cache stores it: already normalised and rotated).  nnc_set_length then
+ * declares how many positions are valid. */
+int nnc_kv_import(nnc_model *model, int32_t layer, int32_t batch_index, const void *k, const void *v,
+                  int32_t n_pos);
+/* Copy the cache of one layer of one sequence, positions [0, n_pos), to k, v (DEVICE, same layout). */
+int nnc_kv_export(nnc_model *model, int32_t layer, int32_t batch_index, void *k, void *v, int32_t n_pos);
+
+int nnc_set_length(nnc_model *model, int32_t n_pos); /* cached positions := n_pos (0 empties the cache) */
+int32_t nnc_get_length(const nnc_model *model);
+
+/* Parity instrumentation.  taps: DEVICE fp32 [n_layers + 1][rows][hidden] (rows = batch for a decode step,
+ * batch * n_tokens for a prefill), receiving the residual stream after the embedding and after every layer of
+ * each following call; NULL switches it off.  While a tap is set, decode steps run kernel by kernel instead
+ * of through the captured graph (same kernels, same order). */
+int nnc_set_hidden_tap(nnc_model *model, float *taps);
+
+/* One decoder layer, one step, batch 1, on a caller-supplied residual-stream vector: x_in, x_out DEVICE fp32
+ * [hidden].  The token sits at position len; its K/V are appended to that layer's cache; len is NOT changed
+ * (call nnc_set_length to advance). */
+int nnc_layer_decode(nnc_model *model, int32_t layer, const float *x_in, float *x_out);
+
+/* Write the ORIGINAL (caller-layout) matrix back from the repacked store: which = 0 wq, 1 wk, 2 wv, 3 wo,
+ * 4 w_gate, 5 w_up, 6 w_down; out DEVICE bf16 of that matrix's shape.  Lets a test check that the repack
+ * loses nothing. */
+int nnc_unrepack(nnc_model *model, int32_t layer, int32_t which, void *out);
+
+/* Reads (and clears) the device status word; synchronises the stream.  0 = no kernel gave up on a wait. */
+int nnc_device_status(nnc_model *model, int32_t *status_out /* HOST */);
+
+/* Number of kernels this library launched on behalf of `model` since creation (graph nodes count once per
+ * graph launch). */
+int64_t nnc_launch_count(const nnc_model *model);
+
+const char *nnc_last_error(const nnc_model *model); /* never NULL; valid until the next call on the model */
+const char *nnc_status_string(int status);
+
+/* ---- single operations, exposed for kernel-level tests and isolated timing ----------------------------
+ * Each runs on `cuda_stream`, allocates nothing, and returns an nnc_status. */
+
+/* y[T][n_out] = X[T][n_in] * W[n_out][n_in]^T on the tensor cores (tcgen05, fp32 accumulation in tensor
+ * memory).  X, W bf16 row-major (n_in contiguous), n_in a multiple of 64, n_out a multiple of 8.
+ * out_f32 != 0: Y is fp32 (and, if accumulate != 0, Y += product); otherwise Y is bf16. */
+int nnc_op_gemm(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                int32_t out_f32, int32_t accumulate, void *cuda_stream);
+/* The same product with the SwiGLU epilogue of the MLP: W rows interleaved (row 2i = gate_i, row 2i+1 = up_i),
+ * Y bf16 [T][n_out/2], Y[t][i] = silu(gate) * up. */
+int nnc_op_gemm_swiglu(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                       void *cuda_stream);
+/* Status word of the nnc_op_* tensor-core kernels (0 = no bounded wait ran out); synchronises the device and
+ * clears the word.  status_out is a HOST pointer. */
+int nnc_op_status(int32_t *status_out);
+
+/* y[n_out] = W[n_out][n_in] x (batch-1 streaming GEMV, fp32 accumulate).  x fp32 [n_in]; y fp32.
+ * If gain != NULL (bf16 [n_in]) x is first RMS-normalised with that gain and eps.
+ * mode 0: y = Wx;  mode 1: y += Wx (residual);  mode 2: rows interleaved gate/up, y[n_out/2] = silu(g)*u. */
+int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t n_in, const void *gain,
+                float eps, int32_t mode, void *cuda_stream);
+
+/* Split-K flash-decode for one query token per sequence over a contiguous cache.
+ *   q fp32 [batch][n_q_heads][128] (already normalised and rotated);  kcache, vcache bf16
+ *   [batch][n_kv_heads][max_seq][128];  n_ctx positions are attended;  out fp32 [batch][n_q_heads][128].
+ *   scratch: DEVICE, at least nnc_attn_scratch_bytes(batch, n_q_heads, n_ctx) bytes, 256-byte aligned. */
+size_t nnc_attn_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t n_ctx);
+int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, float *out, int32_t batch,
+                       int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_ctx, void *scratch,
+                       void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NNC_H_ */

@@ -1,0 +1,159 @@
+// Small row-wise kernels of the forward pass: embedding gather, per-head QK-RMSNorm + RoPE + KV append,
+// row-wise RMSNorm to a bf16 GEMM operand, and the device-side position counter.
+#include "common.cuh"
+#include "nnc_internal.h"
+
+namespace nnc {
+
+namespace {
+
+// x[r][:] = float(E[token_r][:]); one block per row.  Out-of-range ids are clamped.
+__global__ void embed_kernel(const bf16 *__restrict__ E, const int32_t *__restrict__ tokens, float *__restrict__ x,
+                             int H, int vocab, float *__restrict__ tap) {
+    pdl_wait();
+    const int r = blockIdx.x;
+    int tok = tokens[r];
+    tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+    const uint2 *src = reinterpret_cast<const uint2 *>(E + (size_t)tok * H);
+    float4 *dst = reinterpret_cast<float4 *>(x + (size_t)r * H);
+    float4 *tp = tap ? reinterpret_cast<float4 *>(tap + (size_t)r * H) : nullptr;
+    for (int i = threadIdx.x; i < H / 4; i += blockDim.x) {
+        const uint2 u = src[i];
+        const float4 v = make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+        dst[i] = v;
+        if (tp) tp[i] = v;
+    }
+    pdl_launch_dependents();
+}
+
+// One warp per (row, head) of the fused QKV activation [rows][(nq + 2 nkv) * 128] (fp32).
+//   q heads: q <- RoPE_p(RMSNorm_128(q; g_q)) in place (and optionally a bf16 copy for tensor-core attention)
+//   k heads: the same with g_k, then rounded to bf16 into the cache at position p
+//   v heads: rounded to bf16 into the cache at position p
+// p = *d_len + (row % rows_per_seq); sequence = row / rows_per_seq.  Lane l owns elements 2l, 2l+1 and their
+// rotation partners 2l+64, 2l+65 (half-split pairing).
+__global__ void __launch_bounds__(128)
+qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, const bf16 *__restrict__ g_q,
+                           const bf16 *__restrict__ g_k, float eps, const float *__restrict__ rope,
+                           bf16 *__restrict__ kcache, bf16 *__restrict__ vcache, int nq, int nkv, int max_seq,
+                           const int32_t *__restrict__ d_len, bf16 *__restrict__ q_bf16) {
+    pdl_wait();
+    const int heads = nq + 2 * nkv;
+    const int unit = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (unit < rows * heads) {
+        const int row = unit / heads, head = unit % heads;
+        const int seq = row / rows_per_seq;
+        const int pos = *d_len + (row % rows_per_seq);
+        float *p = qkv + (size_t)row * heads * kHeadDim + (size_t)head * kHeadDim;
+        float2 a = reinterpret_cast<float2 *>(p)[lane];        // elements 2l, 2l+1
+        float2 b = reinterpret_cast<float2 *>(p + 64)[lane];   // elements 2l+64, 2l+65
+        if (pos < max_seq) {
+            if (head < nq + nkv) {
+                const bf16 *g = head < nq ? g_q : g_k;
+                const float ss = warp_sum(a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y);
+                const float inv = rsqrtf(ss * (1.f / kHeadDim) + eps);
+                const uint32_t ga = reinterpret_cast<const uint32_t *>(g)[lane];
+                const uint32_t gb = reinterpret_cast<const uint32_t *>(g + 64)[lane];
+                a.x *= inv * bf16_lo(ga); a.y *= inv * bf16_hi(ga);
+                b.x *= inv * bf16_lo(gb); b.y *= inv * bf16_hi(gb);
+                const float4 cs = reinterpret_cast<const float4 *>(rope + (size_t)pos * kHeadDim)[lane];  // c0 s0 c1 s1
+                const float2 ra = make_float2(a.x * cs.x - b.x * cs.y, a.y * cs.z - b.y * cs.w);
+                const float2 rb = make_float2(b.x * cs.x + a.x * cs.y, b.y * cs.z + a.y * cs.w);
+                a = ra; b = rb;
+            }
+            if (head < nq) {
+                reinterpret_cast<float2 *>(p)[lane] = a;
+                reinterpret_cast<float2 *>(p + 64)[lane] = b;
+                if (q_bf16) {
+                    bf16 *qb = q_bf16 + ((size_t)row * nq + head) * kHeadDim;
+                    reinterpret_cast<uint32_t *>(qb)[lane] = pack_bf16x2(a.x, a.y);
+                    reinterpret_cast<uint32_t *>(qb + 64)[lane] = pack_bf16x2(b.x, b.y);
+                }
+            } else {
+                const bool is_k = head < nq + nkv;
+                const int j = is_k ? head - nq : head - nq - nkv;
+                bf16 *dst = (is_k ? kcache : vcache) + (((size_t)seq * nkv + j) * max_seq + pos) * kHeadDim;
+                reinterpret_cast<uint32_t *>(dst)[lane] = pack_bf16x2(a.x, a.y);
+                reinterpret_cast<uint32_t *>(dst + 64)[lane] = pack_bf16x2(b.x, b.y);
+            }
+        }
+    }
+    pdl_launch_dependents();
+}
+
+// out[i][:] = bf16(RMSNorm(x[first + i*step][:]; gain)); one block per output row.
+__global__ void __launch_bounds__(256)
+rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out, int H, float eps,
+                    int first, int step) {
+    __shared__ float red[8];
+    pdl_wait();
+    const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
+    uint2 *dst = reinterpret_cast<uint2 *>(out + (size_t)blockIdx.x * H);
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < H / 4; i += 256) {
+        const float4 v = src[i];
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)H + eps);
+    for (int i = threadIdx.x; i < H / 4; i += 256) {
+        const float4 v = src[i];
+        const uint2 g = reinterpret_cast<const uint2 *>(gain)[i];
+        uint2 o;
+        o.x = pack_bf16x2(v.x * inv * bf16_lo(g.x), v.y * inv * bf16_hi(g.x));
+        o.y = pack_bf16x2(v.z * inv * bf16_lo(g.y), v.w * inv * bf16_hi(g.y));
+        dst[i] = o;
+    }
+    pdl_launch_dependents();
+}
+
+__global__ void copy_f32_kernel(const float *__restrict__ src, float *__restrict__ dst, size_t n) {
+    pdl_wait();
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+    pdl_launch_dependents();
+}
+
+__global__ void add_len_kernel(int32_t *d_len, int delta) {
+    pdl_wait();
+    if (threadIdx.x == 0) *d_len += delta;
+}
+
+}  // namespace
+
+cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
+                         int vocab, float *tap) {
+    return launch(lc, embed_kernel, dim3(rows), dim3(128), E, tokens, x, H, vocab, tap);
+}
+
+cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
+                                       const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
+                                       bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
+                                       const int32_t *d_len, bf16 *q_bf16_out) {
+    const long units = (long)rows * (nq + 2 * nkv);
+    return launch(lc, qk_norm_rope_append_kernel, dim3((unsigned)((units + 3) / 4)), dim3(128), qkv, rows,
+                  rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, q_bf16_out);
+}
+
+cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, int rows, int H,
+                                float eps, int first, int step) {
+    return launch(lc, rmsnorm_rows_kernel, dim3(rows), dim3(256), x, gain, out, H, eps, first, step);
+}
+
+cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n) {
+    size_t blocks = (n + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    return launch(lc, copy_f32_kernel, dim3((unsigned)blocks), dim3(256), src, dst, n);
+}
+
+cudaError_t launch_add_len(const LaunchCtx &lc, int32_t *d_len, int delta) {
+    return launch(lc, add_len_kernel, dim3(1), dim3(32), d_len, delta);
+}
+
+}  // namespace nnc

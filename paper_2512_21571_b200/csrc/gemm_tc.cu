@@ -1,0 +1,432 @@
+// Tensor-core GEMM for the prompt phase and batched decode:  Y[T][N] = X[T][K] * W[N][K]^T, bf16 operands,
+// fp32 accumulation in tensor memory (tcgen05 / TMEM), hand-written PTX.
+//
+// Structure (one persistent CTA per SM, 192 threads):
+//   warp 0      TMA producer: streams 128-row x 64-column (128-byte, 128B-swizzled) operand tiles into a
+//               shared-memory ring, one mbarrier per stage
+//   warp 1      MMA issuer: one elected lane issues tcgen05.mma (M=128, N=BN, K=16) four times per stage and
+//               commits the stage back to the producer; accumulators alternate between two TMEM buffers
+//   warps 2-5   epilogue: tcgen05.ld 32 columns at a time, apply the epilogue, store; runs concurrently with
+//               the main loop of the next tile thanks to the second accumulator
+// Two operand assignments share the code: tokens on the M side (prefill; weights are the N operand, BN=256)
+// or weights on the M side ("swap", used when there are few tokens, e.g. a decode batch of 32: weights fill
+// the 128 TMEM lanes and the tokens are the narrow N operand, so no tensor-core work is wasted on padding).
+// Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA raises an abort flag, records a
+// status word for the host, drains and frees its TMEM.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "nnc_internal.h"
+
+namespace nnc {
+
+namespace {
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;
+constexpr int kGemmThreads = 192;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false if the limit ran out or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          int code) {
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes (64 elements) with the
+// 128-byte swizzle TMA applied: 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1,
+// layout type 2 (128B swizzle).  Advancing K by 16 elements inside the swizzle atom adds 32 bytes to the start.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;            // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset
+    d |= (uint64_t)1 << 46;            // descriptor version
+    d |= (uint64_t)2 << 61;            // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+struct GemmParams {
+    void *Y;          // output
+    int T, N, K;      // tokens, weight rows, reduction
+    int ldy;          // output row stride in elements
+    int m_tiles, n_tiles;
+    int *status;
+};
+
+template <int BN>
+struct SmemLayout {
+    static constexpr int kStageA = kBM * kBK * 2;
+    static constexpr int kStageB = BN * kBK * 2;
+    static constexpr int kStage = kStageA + kStageB;
+    static constexpr int kStages = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr int kBytes = kStages * kStage + 1024 /*align slack*/ + 256 /*barriers*/;
+    static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
+};
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
+
+// EPI: 0 fp32 store, 1 bf16 store, 2 fp32 accumulate (Y += D), 3 SwiGLU on interleaved gate/up weight rows -> bf16
+template <int BN, bool SWAP, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant__ CUtensorMap map_n, GemmParams p) {
+    using L = SmemLayout<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + L::kStages * L::kStage;      // full[S], empty[S], tfull[2], tempty[2], 8 B each
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (L::kStages + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * L::kStages + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * L::kStages + 2 + a); };
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &abort_s;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+                     "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int kb_count = p.K / kBK;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        if (lane == 0) {  // ---------------- TMA producer ----------------
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(stage), L::kStage);
+                    const uint32_t sa = base + stage * L::kStage;
+                    tma_load_2d(sa, &map_m, full_bar(stage), kb * kBK, mt * kBM);
+                    tma_load_2d(sa + L::kStageA, &map_n, full_bar(stage), kb * kBK, nt * BN);
+                    if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {  // ---------------- MMA issuer ----------------
+            constexpr uint32_t idesc = make_idesc(BN);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * L::kStage;
+                    const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + L::kStageA);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)
+                        umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                    umma_commit(empty_bar(stage));
+                    if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {  // ---------------- epilogue warps 2..5 ----------------
+        const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
+            tc_fence_after();
+            const int m = mt * kBM + quarter * 32 + lane;  // D row held by this thread
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                const int n0 = nt * BN + c0;
+                if (!SWAP) {
+                    // row m = token, columns n0.. = weight rows: contiguous per thread
+                    if (m < p.T) {
+                        if (EPI == 3) {
+                            bf16 *y = reinterpret_cast<bf16 *>(p.Y) + (size_t)m * p.ldy + (n0 >> 1);
+                            if (n0 + 32 <= p.N) {
+                                uint32_t o[8];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    o[i] = pack_bf16x2(silu_mul(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])),
+                                                       silu_mul(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])));
+                                reinterpret_cast<uint4 *>(y)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                                reinterpret_cast<uint4 *>(y)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                            } else {
+                                for (int i = 0; i < 16; ++i)
+                                    if (n0 + 2 * i + 1 < p.N)
+                                        y[i] = __float2bfloat16_rn(silu_mul(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])));
+                            }
+                        } else if (EPI == 1) {
+                            bf16 *y = reinterpret_cast<bf16 *>(p.Y) + (size_t)m * p.ldy + n0;
+                            if (n0 + 32 <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    uint4 o;
+                                    o.x = pack_bf16x2(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1]));
+                                    o.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
+                                    o.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
+                                    o.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
+                                    reinterpret_cast<uint4 *>(y)[i] = o;
+                                }
+                            } else {
+                                for (int i = 0; i < 32; ++i)
+                                    if (n0 + i < p.N) y[i] = __float2bfloat16_rn(__uint_as_float(r[i]));
+                            }
+                        } else {
+                            float *y = reinterpret_cast<float *>(p.Y) + (size_t)m * p.ldy + n0;
+                            if (n0 + 32 <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    float4 v = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                                           __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                                    if (EPI == 2) {
+                                        const float4 o = reinterpret_cast<float4 *>(y)[i];
+                                        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                                    }
+                                    reinterpret_cast<float4 *>(y)[i] = v;
+                                }
+                            } else {
+                                for (int i = 0; i < 32; ++i)
+                                    if (n0 + i < p.N) y[i] = (EPI == 2 ? y[i] : 0.f) + __uint_as_float(r[i]);
+                            }
+                        }
+                    }
+                } else {
+                    // row m = weight row, columns = tokens: a warp stores 32 consecutive weight rows per token
+                    if (EPI == 3) {
+                        // gate in even lanes, up in odd lanes
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float mine = __uint_as_float(r[i]);
+                            const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                            const int t = n0 + i;
+                            if (!(lane & 1) && m + 1 < p.N && t < p.T)
+                                reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + (m >> 1)] = __float2bfloat16_rn(silu_mul(mine, other));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int t = n0 + i;
+                            if (m < p.N && t < p.T) {
+                                const float v = __uint_as_float(r[i]);
+                                if (EPI == 1) reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + m] = __float2bfloat16_rn(v);
+                                else if (EPI == 2) reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] += v;
+                                else reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] = v;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---- teardown ----
+    __syncwarp();
+    if (*abort_flag && threadIdx.x == 0) {
+        // let copies that are still in flight land before the shared memory is released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][K], K contiguous; box = 64 columns (128 bytes) x box_rows, 128-byte swizzle, zero fill
+bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, bool SWAP, int EPI>
+cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
+                      int *status) {
+    using L = SmemLayout<BN>;
+    auto kern = gemm_tc_kernel<BN, SWAP, EPI>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    CUtensorMap map_m, map_n;
+    GemmParams p;
+    p.Y = Y; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status;
+    if (!SWAP) {
+        if (!make_map(&map_m, X, T, K, kBM) || !make_map(&map_n, W, N, K, BN)) return cudaErrorInvalidValue;
+        p.m_tiles = (T + kBM - 1) / kBM;
+        p.n_tiles = (N + BN - 1) / BN;
+    } else {
+        if (!make_map(&map_m, W, N, K, kBM) || !make_map(&map_n, X, T, K, BN)) return cudaErrorInvalidValue;
+        p.m_tiles = (N + kBM - 1) / kBM;
+        p.n_tiles = (T + BN - 1) / BN;
+    }
+    int grid = p.m_tiles * p.n_tiles;
+    if (grid > lc.sm_count) grid = lc.sm_count;
+    if (lc.launches) ++*lc.launches;
+    kern<<<grid, kGemmThreads, L::kBytes, lc.stream>>>(map_m, map_n, p);
+    return cudaGetLastError();
+}
+
+template <int EPI>
+cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
+                     int *status) {
+    if (T <= 32) return launch_tc<32, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
+    if (T <= 64) return launch_tc<64, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
+    if (T <= 128) return launch_tc<128, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
+    return launch_tc<256, false, EPI>(lc, X, W, Y, T, N, K, ldy, status);
+}
+
+}  // namespace
+
+bool gemm_tc_available() { return get_encode() != nullptr; }
+
+// Y[T][*] (row stride ldy) = epilogue(X[T][K] * W[N][K]^T).  X, W 16-byte aligned, K % 64 == 0.
+cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
+                        int epi, int *status) {
+    if (T <= 0 || N <= 0 || K <= 0 || K % kBK != 0 || N % 8 != 0) return cudaErrorInvalidValue;
+    if (((uintptr_t)X | (uintptr_t)W | (uintptr_t)Y) & 15) return cudaErrorInvalidValue;
+    switch (epi) {
+        case kEpiStoreF32: return dispatch<0>(lc, X, W, Y, T, N, K, ldy, status);
+        case kEpiStoreBf16: return dispatch<1>(lc, X, W, Y, T, N, K, ldy, status);
+        case kEpiAccumF32: return dispatch<2>(lc, X, W, Y, T, N, K, ldy, status);
+        case kEpiSwigluBf16: return dispatch<3>(lc, X, W, Y, T, N, K, ldy, status);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace nnc

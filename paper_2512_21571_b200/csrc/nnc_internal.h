@@ -1,0 +1,83 @@
+// Host-side internals of libnnc: launch context, kernel launchers, and the launch helper they share.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/nnc.h"
+
+namespace nnc {
+
+typedef __nv_bfloat16 bf16;
+
+struct LaunchCtx {
+    cudaStream_t stream;
+    int sm_count;
+    bool pdl;           // launch with programmatic stream serialization (kernels call pdl_wait themselves)
+    int64_t *launches;  // bumped once per kernel launch (may be null)
+};
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch(const LaunchCtx &lc, void (*kern)(KArgs...), dim3 grid, dim3 block, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    if (lc.launches) ++*lc.launches;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// ---- decode GEMV family (decode_gemv.cu) --------------------------------------------------------------
+enum GemvMode { kGemvStore = 0, kGemvResidual = 1, kGemvSwiglu = 2, kGemvLogits = 3 };
+
+constexpr int kArgmaxMaxBlocks = 4096;
+struct ArgmaxScratch {
+    float *part_val;    // [kArgmaxMaxBlocks]
+    int32_t *part_idx;  // [kArgmaxMaxBlocks]
+    uint32_t *ticket;   // one counter, zero between launches
+    int32_t *out;       // result; null = no arg-max
+};
+
+cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
+                        const bf16 *gain, float eps, int mode, const ArgmaxScratch *am);
+
+// ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
+cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
+                         int vocab, float *tap);
+cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
+                                       const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
+                                       bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
+                                       const int32_t *d_len, bf16 *q_bf16_out);
+cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, int rows, int H,
+                                float eps, int first, int step);
+cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n);
+cudaError_t launch_add_len(const LaunchCtx &lc, int32_t *d_len, int delta);
+
+// ---- attention ----------------------------------------------------------------------------------------
+constexpr int kAttnMaxSplits = 64;
+int attn_decode_splits(int sm_count, int batch, int nkv, int max_ctx);
+size_t attn_decode_scratch_floats(int batch, int nq, int n_splits);
+cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, const bf16 *kcache,
+                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, int out_row_stride, float *part,
+                               uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
+                               int max_seq, int n_splits);
+cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
+                                const bf16 *vcache, bf16 *out, int nq, int nkv, int max_seq, const int32_t *d_len);
+
+// ---- GEMM (gemm_tc.cu) --------------------------------------------------------------------------------
+enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwigluBf16 = 3 };
+bool gemm_tc_available();
+cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
+                        int epi, int *status);
+
+// ---- repack (repack.cu) -------------------------------------------------------------------------------
+// dst rows [row0, row0 + rows) <- src rows [0, rows), row length K (plain row copy into a taller matrix)
+cudaError_t launch_copy_rows(const LaunchCtx &lc, const bf16 *src, bf16 *dst, int rows, int K, int dst_row0,
+                             int dst_row_step, int src_row0, int src_row_step);
+
+}  // namespace nnc

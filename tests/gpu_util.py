@@ -1,0 +1,28 @@
+"""Helpers for the GPU parity tests: build the CUDA model and the oracle from the same seeded weights."""
+import torch
+
+from paper_2512_21571_b200 import synth
+
+
+def to_cpu(w: dict) -> dict:
+    c = lambda t: None if t is None else t.cpu().contiguous()
+    return {"embed": c(w["embed"]), "lm_head": c(w.get("lm_head")), "g_final": c(w["g_final"]),
+            "layers": [{k: c(v) for k, v in lw.items()} for lw in w["layers"]]}
+
+
+def make_pair(oracle_mod, shape, seed, max_seq, max_batch=1, max_tokens=None, gains=False, sigma=0.02):
+    """(cuda model, oracle, gpu weights).  Weights are generated once on the GPU and copied to the host."""
+    from paper_2512_21571_b200 import binding
+    w = synth.make_weights(shape, seed, device="cuda", sigma=sigma)
+    if gains:
+        synth.random_gains(w, seed + 1)
+    m = binding.Model(shape, w, max_seq=max_seq, max_batch=max_batch, max_tokens=max_tokens)
+    o = oracle_mod.Oracle(shape, to_cpu(w), max_seq=max_seq)
+    return m, o, w
+
+
+def rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
+    """max over rows of ||a - b|| / ||b|| (b = oracle)."""
+    a, b = a.double().cpu(), b.double().cpu()
+    a, b = a.reshape(-1, a.shape[-1]), b.reshape(-1, b.shape[-1])
+    return ((a - b).norm(dim=-1) / b.norm(dim=-1)).max().item()

@@ -1,0 +1,119 @@
+"""Kernel-level parity: each CUDA operation, called through the C ABI, against the oracle's matching function
+on the same seeded inputs.  Sizes span several tiles and ragged tails."""
+import math
+
+import pytest
+import torch
+
+from paper_2512_21571_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nnc():
+    from paper_2512_21571_b200 import binding
+    return binding
+
+
+def _w(seed, stream, shape, sigma=0.02):
+    return synth.normal(seed, stream, shape, sigma, torch.bfloat16, "cuda")
+
+
+@pytest.mark.parametrize("n_out,n_in", [(8, 64), (1000, 384), (4096, 1024), (6144, 4096), (1024, 3072), (2050, 640)])
+def test_gemv_store_and_residual(nnc, oracle_mod, n_out, n_in):
+    W = _w(1, 1, (n_out, n_in))
+    x = synth.normal(1, 2, (n_in,), 1.0, torch.float32, "cuda")
+    want = oracle_mod.matmul(W.cpu(), x.cpu().view(1, -1))[0]
+    y = nnc.op_gemv(W, x, mode=0)
+    assert torch.allclose(y.cpu(), want, rtol=1e-4, atol=2e-5 * math.sqrt(n_in))
+    base = synth.normal(1, 3, (n_out,), 1.0, torch.float32, "cuda")
+    y2 = nnc.op_gemv(W, x, mode=1, y=base.clone())
+    assert torch.allclose(y2.cpu(), base.cpu() + want, rtol=1e-4, atol=2e-5 * math.sqrt(n_in))
+
+
+@pytest.mark.parametrize("n_out,n_in", [(1024, 256), (6144, 1024), (24576, 4096), (1280, 384)])
+def test_gemv_norm_prologue_and_swiglu(nnc, oracle_mod, n_out, n_in):
+    W = _w(2, 1, (n_out, n_in))
+    x = synth.normal(2, 2, (n_in,), 3.0, torch.float32, "cuda")
+    gain = (1.0 + synth.normal(2, 3, (n_in,), 0.1, torch.float32, "cuda")).to(torch.bfloat16)
+    h = oracle_mod.rmsnorm(x.cpu(), gain.cpu(), 1e-6)
+    # rows interleaved gate/up
+    full = oracle_mod.matmul(W.cpu(), h.view(1, -1))[0]
+    y = nnc.op_gemv(W, x, mode=0, gain=gain, eps=1e-6)
+    assert torch.allclose(y.cpu(), full, rtol=1e-4, atol=1e-4)
+    want = torch.tensor([oracle_mod.silu(float(g)) * float(u) for g, u in zip(full[0::2], full[1::2])])
+    a = nnc.op_gemv(W, x, mode=2, gain=gain, eps=1e-6)
+    assert a.shape == (n_out // 2,)
+    assert torch.allclose(a.cpu(), want, rtol=1e-4, atol=1e-5)
+
+
+def test_gemv_identity_and_one_hot(nnc):
+    n = 256
+    eye = torch.eye(n, dtype=torch.bfloat16, device="cuda")
+    x = synth.normal(3, 1, (n,), 1.0, torch.float32, "cuda")
+    assert torch.equal(nnc.op_gemv(eye, x), x)
+    W = _w(3, 2, (512, n))
+    e = torch.zeros(n, device="cuda"); e[37] = 1.0
+    assert torch.equal(nnc.op_gemv(W, e), W[:, 37].float())
+
+
+@pytest.mark.parametrize("T,N,K", [(1, 256, 64), (7, 384, 256), (32, 1024, 256), (33, 1000, 640), (64, 512, 128),
+                                   (100, 2048, 1024), (128, 256, 64), (129, 1280, 384), (300, 6144, 1024),
+                                   (1000, 1000, 512), (513, 24576, 256)])
+def test_gemm_tensor_core_against_oracle_matmul(nnc, oracle_mod, T, N, K):
+    X = synth.normal(4, 1, (T, K), 1.0, torch.bfloat16, "cuda")
+    W = _w(4, 2, (N, K))
+    Y = nnc.op_gemm(X, W, out_f32=True)
+    torch.cuda.synchronize()
+    assert nnc.op_status() == 0
+    rows = sorted(set([0, T - 1, T // 2] + list(range(0, T, max(1, T // 5)))))
+    want = oracle_mod.matmul(W.cpu(), X[rows].float().cpu())
+    assert torch.allclose(Y[rows].cpu(), want, rtol=1e-4, atol=2e-5 * math.sqrt(K))
+    # every element against a float64 product on the device (same operands), to catch misplaced tiles
+    ref = (X.double() @ W.double().T)
+    assert (Y.double() - ref).abs().max().item() < 2e-5 * math.sqrt(K)
+    Yb = nnc.op_gemm(X, W, out_f32=False)
+    assert torch.allclose(Yb.float(), ref.float(), rtol=1e-2, atol=1e-3)
+    acc = synth.normal(4, 3, (T, N), 1.0, torch.float32, "cuda")
+    Y2 = nnc.op_gemm(X, W, accumulate_into=acc.clone())
+    assert (Y2.double() - (acc.double() + ref)).abs().max().item() < 1e-4 * math.sqrt(K)
+    assert nnc.op_status() == 0
+
+
+@pytest.mark.parametrize("T,N,K", [(5, 512, 256), (64, 1024, 128), (130, 1280, 384), (400, 6144, 1024)])
+def test_gemm_swiglu_epilogue(nnc, oracle_mod, T, N, K):
+    X = synth.normal(5, 1, (T, K), 1.0, torch.bfloat16, "cuda")
+    W = _w(5, 2, (N, K), sigma=0.1)
+    A = nnc.op_gemm_swiglu(X, W)
+    rows = [0, T - 1, T // 3]
+    full = oracle_mod.matmul(W.cpu(), X[rows].float().cpu())
+    g, u = full[:, 0::2], full[:, 1::2]
+    want = g / (1 + torch.exp(-g)) * u
+    assert A.shape == (T, N // 2)
+    assert torch.allclose(A[rows].float().cpu(), want, rtol=1e-2, atol=2e-3)
+    ref = X.double() @ W.double().T
+    refa = (ref[:, 0::2] / (1 + torch.exp(-ref[:, 0::2])) * ref[:, 1::2]).float()
+    assert torch.allclose(A.float(), refa, rtol=1e-2, atol=2e-3)
+    assert nnc.op_status() == 0
+
+
+@pytest.mark.parametrize("batch,nq,nkv,n_ctx,max_seq", [(1, 2, 1, 1, 8), (1, 16, 8, 129, 256), (2, 4, 4, 17, 64),
+                                                         (1, 32, 8, 4097, 4224), (3, 8, 1, 1000, 1024),
+                                                         (1, 16, 8, 777, 8192)])
+def test_attn_decode_against_oracle(nnc, oracle_mod, batch, nq, nkv, n_ctx, max_seq):
+    q = synth.normal(6, 1, (batch, nq, 128), 1.0, torch.float32, "cuda")
+    kc = synth.normal(6, 2, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    vc = synth.normal(6, 3, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    # positions beyond n_ctx hold NaN bit patterns: they must never be read into the result
+    kc[:, :, n_ctx:] = float("nan"); vc[:, :, n_ctx:] = float("nan")
+    out = nnc.op_attn_decode(q, kc, vc, n_ctx)
+    out2 = nnc.op_attn_decode(q, kc, vc, n_ctx)
+    assert torch.equal(out, out2), "split-K combine must not depend on arrival order"
+    G = nq // nkv
+    qc, kcc, vcc = q.cpu(), kc.cpu(), vc.cpu()
+    for b in range(batch):
+        for i in sorted(set([0, nq - 1, nq // 2])):
+            want = oracle_mod.attend(qc[b, i], kcc[b, i // G, :n_ctx].contiguous(), vcc[b, i // G, :n_ctx].contiguous())
+            assert torch.allclose(out[b, i].cpu(), want, rtol=1e-4, atol=2e-5), (b, i)
+    assert torch.isfinite(out).all()
