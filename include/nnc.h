@@ -56,6 +56,11 @@ typedef struct {
     int32_t tie_embeddings; /* 1: the lm_head is the embedding matrix */
     float rms_eps;          /* 1e-6 for Qwen3 */
     float rope_theta;       /* 1e6 for Qwen3 */
+    int32_t fast_bf16_activations; /* tensor-core path only (prompt phase, batched decode).  0 (default): each
+                             * activation operand is fed as two bf16 terms, value + rounding residual, i.e. ~16
+                             * mantissa bits, which keeps deep models inside the parity tolerance at twice the
+                             * tensor-core work.  1: one bf16 term (half the tensor-core work; rounding error of
+                             * 2^-9 per operand accumulates to a few percent over ~30 layers). */
 } nnc_config;
 
 /* Per-layer weights: DEVICE pointers, bf16.  Read only during nnc_model_create (they are repacked into the
@@ -154,15 +159,17 @@ const char *nnc_status_string(int status);
 /* ---- single operations, exposed for kernel-level tests and isolated timing ----------------------------
  * Each runs on `cuda_stream`, allocates nothing, and returns an nnc_status. */
 
-/* y[T][n_out] = X[T][n_in] * W[n_out][n_in]^T on the tensor cores (tcgen05, fp32 accumulation in tensor
- * memory).  X, W bf16 row-major (n_in contiguous), n_in a multiple of 64, n_out a multiple of 8.
+/* y[T][n_out] = (X + X_lo)[T][n_in] * W[n_out][n_in]^T on the tensor cores (tcgen05, fp32 accumulation in
+ * tensor memory).  X, W bf16 row-major (n_in contiguous), n_in a multiple of 64, n_out a multiple of 8.
+ * X_lo: NULL, or a second bf16 [T][n_in] matrix (the rounding residual of the activations) multiplied with
+ * the same weights into the same accumulator.
  * out_f32 != 0: Y is fp32 (and, if accumulate != 0, Y += product); otherwise Y is bf16. */
-int nnc_op_gemm(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+int nnc_op_gemm(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
                 int32_t out_f32, int32_t accumulate, void *cuda_stream);
 /* The same product with the SwiGLU epilogue of the MLP: W rows interleaved (row 2i = gate_i, row 2i+1 = up_i),
- * Y bf16 [T][n_out/2], Y[t][i] = silu(gate) * up. */
-int nnc_op_gemm_swiglu(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
-                       void *cuda_stream);
+ * Y bf16 [T][n_out/2], Y[t][i] = silu(gate) * up; n_out a multiple of 16 (rows of Y stay 16-byte aligned). */
+int nnc_op_gemm_swiglu(const void *X, const void *X_lo, const void *W, void *Y, void *Y_lo, int32_t T,
+                       int32_t n_out, int32_t n_in, void *cuda_stream); /* Y_lo: NULL or the residual of Y */
 /* Status word of the nnc_op_* tensor-core kernels (0 = no bounded wait ran out); synchronises the device and
  * clears the word.  status_out is a HOST pointer. */
 int nnc_op_status(int32_t *status_out);

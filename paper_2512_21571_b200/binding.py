@@ -24,7 +24,7 @@ lib = C.CDLL(LIB_PATH)
 class nnc_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "intermediate",
                                          "vocab", "max_seq", "max_batch", "max_tokens", "tie_embeddings")] + \
-               [("rms_eps", C.c_float), ("rope_theta", C.c_float)]
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("fast_bf16_activations", C.c_int32)]
 
 
 LAYER_FIELDS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "g_in", "g_post", "g_q", "g_k")
@@ -59,9 +59,10 @@ EXPORTS = {
     "nnc_launch_count": (C.c_int64, [C.c_void_p]),
     "nnc_last_error": (C.c_char_p, [C.c_void_p]),
     "nnc_status_string": (C.c_char_p, [C.c_int]),
-    "nnc_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                              C.c_void_p]),
-    "nnc_op_gemm_swiglu": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
+    "nnc_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                              C.c_int32, C.c_void_p]),
+    "nnc_op_gemm_swiglu": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                     C.c_int32, C.c_void_p]),
     "nnc_op_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "nnc_op_gemv": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_float, C.c_int32,
                               C.c_void_p]),
@@ -92,12 +93,14 @@ def _dev(t: torch.Tensor, dtype) -> int:
 class Model:
     """nnc_model_create / nnc_prefill / nnc_decode_step and the auxiliary calls, one method per C function."""
 
-    def __init__(self, shape, weights: dict, max_seq: int, max_batch: int = 1, max_tokens: Optional[int] = None):
+    def __init__(self, shape, weights: dict, max_seq: int, max_batch: int = 1, max_tokens: Optional[int] = None,
+                 fast_bf16_activations: bool = False):
         self.shape = shape
         self.cfg = nnc_config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                               shape.intermediate, shape.vocab, max_seq, max_batch,
                               max_tokens if max_tokens is not None else max(max_batch, 1),
-                              int(shape.tie_embeddings), shape.rms_eps, shape.rope_theta)
+                              int(shape.tie_embeddings), shape.rms_eps, shape.rope_theta,
+                              int(fast_bf16_activations))
         self.handle = C.c_void_p()
         nbytes = lib.nnc_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
@@ -215,25 +218,35 @@ def _ok(rc: int, what: str):
         raise NncError(rc, what)
 
 
-def op_gemm(X: torch.Tensor, W: torch.Tensor, out_f32: bool = True, accumulate_into: Optional[torch.Tensor] = None):
+def split_bf16(x: torch.Tensor):
+    """fp32 -> (hi, lo) bf16 pair with hi + lo ~ x to 16 mantissa bits (input marshalling for op_gemm)."""
+    hi = x.to(torch.bfloat16)
+    return hi, (x - hi.float()).to(torch.bfloat16)
+
+
+def op_gemm(X: torch.Tensor, W: torch.Tensor, out_f32: bool = True, accumulate_into: Optional[torch.Tensor] = None,
+            X_lo: Optional[torch.Tensor] = None):
     T, K = X.shape
     N = W.shape[0]
     if accumulate_into is not None:
         Y = accumulate_into
     else:
         Y = torch.empty(T, N, dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
-    _ok(lib.nnc_op_gemm(_dev(X, torch.bfloat16), _dev(W, torch.bfloat16), Y.data_ptr(), T, N, K, int(out_f32),
+    _ok(lib.nnc_op_gemm(_dev(X, torch.bfloat16), _dev(X_lo, torch.bfloat16) if X_lo is not None else None,
+                        _dev(W, torch.bfloat16), Y.data_ptr(), T, N, K, int(out_f32),
                         int(accumulate_into is not None), _stream_ptr()), "nnc_op_gemm")
     return Y
 
 
-def op_gemm_swiglu(X: torch.Tensor, W: torch.Tensor):
+def op_gemm_swiglu(X: torch.Tensor, W: torch.Tensor, X_lo: Optional[torch.Tensor] = None, want_lo: bool = False):
     T, K = X.shape
     N = W.shape[0]
     Y = torch.empty(T, N // 2, dtype=torch.bfloat16, device="cuda")
-    _ok(lib.nnc_op_gemm_swiglu(_dev(X, torch.bfloat16), _dev(W, torch.bfloat16), Y.data_ptr(), T, N, K, _stream_ptr()),
-        "nnc_op_gemm_swiglu")
-    return Y
+    Y_lo = torch.empty_like(Y) if want_lo else None
+    _ok(lib.nnc_op_gemm_swiglu(_dev(X, torch.bfloat16), _dev(X_lo, torch.bfloat16) if X_lo is not None else None,
+                               _dev(W, torch.bfloat16), Y.data_ptr(), Y_lo.data_ptr() if want_lo else None, T, N, K,
+                               _stream_ptr()), "nnc_op_gemm_swiglu")
+    return (Y, Y_lo) if want_lo else Y
 
 
 def op_status() -> int:

@@ -27,7 +27,7 @@ template <int G>
 __global__ void __launch_bounds__(128)
 attn_decode_kernel(const float *__restrict__ q, int q_row_stride, const bf16 *__restrict__ kcache,
                    const bf16 *__restrict__ vcache, float *__restrict__ out_f32, bf16 *__restrict__ out_bf16,
-                   int out_row_stride, float *__restrict__ part, uint32_t *__restrict__ tickets,
+                   bf16 *__restrict__ out_bf16_lo, int out_row_stride, float *__restrict__ part, uint32_t *__restrict__ tickets,
                    const int32_t *__restrict__ d_len, int len_add, int nkv, int max_seq, int n_splits) {
     __shared__ float sc[G][kTile];       // scores, then probabilities, of the current tile
     __shared__ float red[4][G][kHeadDim];
@@ -196,7 +196,11 @@ attn_decode_kernel(const float *__restrict__ q, int q_row_stride, const bf16 *__
         const float r = o / L;
         const size_t oi = (size_t)b * out_row_stride + (size_t)(j * G + g) * kHeadDim + tid;
         if (out_f32) out_f32[oi] = r;
-        if (out_bf16) out_bf16[oi] = __float2bfloat16_rn(r);
+        if (out_bf16) {
+            const bf16 hi = __float2bfloat16_rn(r);
+            out_bf16[oi] = hi;
+            if (out_bf16_lo) out_bf16_lo[oi] = __float2bfloat16_rn(r - __bfloat162float(hi));
+        }
     }
     if (tid == 0) tickets[b * nkv + j] = 0u;
 }
@@ -218,7 +222,8 @@ size_t attn_decode_scratch_floats(int batch, int nq, int n_splits) {
 }
 
 cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, const bf16 *kcache,
-                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, int out_row_stride, float *part,
+                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride,
+                               float *part,
                                uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
                                int max_seq, int n_splits) {
     const int G = nq / nkv;
@@ -226,7 +231,7 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
 #define NNC_ATTN_CASE(GG)                                                                                       \
     case GG:                                                                                                    \
         return launch(lc, attn_decode_kernel<GG>, grid, block, q, q_row_stride, kcache, vcache, out_f32,       \
-                      out_bf16, out_row_stride, part, tickets, d_len, len_add, nkv, max_seq, n_splits);
+                      out_bf16, out_bf16_lo, out_row_stride, part, tickets, d_len, len_add, nkv, max_seq, n_splits);
     switch (G) {
         NNC_ATTN_CASE(1)
         NNC_ATTN_CASE(2)

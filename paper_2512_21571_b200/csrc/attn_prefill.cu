@@ -13,8 +13,8 @@ namespace {
 
 __global__ void __launch_bounds__(128)
 attn_prefill_kernel(const float *__restrict__ qkv, int rows, int rows_per_seq, const bf16 *__restrict__ kcache,
-                    const bf16 *__restrict__ vcache, bf16 *__restrict__ out, int nq, int nkv, int max_seq,
-                    const int32_t *__restrict__ d_len) {
+                    const bf16 *__restrict__ vcache, bf16 *__restrict__ out, bf16 *__restrict__ out_lo, int nq, int nkv,
+                    int max_seq, const int32_t *__restrict__ d_len) {
     __shared__ __align__(16) float qs[4][kHeadDim];
     pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -75,16 +75,24 @@ attn_prefill_kernel(const float *__restrict__ qkv, int rows, int rows_per_seq, c
     uint2 o;
     o.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
     o.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-    reinterpret_cast<uint2 *>(out + (size_t)row * nq * kHeadDim + (size_t)head * kHeadDim)[lane] = o;
+    const size_t oi = (size_t)row * nq * kHeadDim + (size_t)head * kHeadDim;
+    reinterpret_cast<uint2 *>(out + oi)[lane] = o;
+    if (out_lo) {  // rounding residual: out + out_lo carries 16 mantissa bits
+        uint2 r;
+        r.x = pack_bf16x2(acc[0] * inv - bf16_lo(o.x), acc[1] * inv - bf16_hi(o.x));
+        r.y = pack_bf16x2(acc[2] * inv - bf16_lo(o.y), acc[3] * inv - bf16_hi(o.y));
+        reinterpret_cast<uint2 *>(out_lo + oi)[lane] = r;
+    }
 }
 
 }  // namespace
 
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
-                                const bf16 *vcache, bf16 *out, int nq, int nkv, int max_seq, const int32_t *d_len) {
+                                const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
+                                const int32_t *d_len) {
     const long units = (long)rows * nq;
     return launch(lc, attn_prefill_kernel, dim3((unsigned)((units + 3) / 4)), dim3(128), qkv, rows, rows_per_seq,
-                  kcache, vcache, out, nq, nkv, max_seq, d_len);
+                  kcache, vcache, out, out_lo, nq, nkv, max_seq, d_len);
 }
 
 }  // namespace nnc

@@ -82,10 +82,11 @@ qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, 
     pdl_launch_dependents();
 }
 
-// out[i][:] = bf16(RMSNorm(x[first + i*step][:]; gain)); one block per output row.
+// out[i][:] = bf16(RMSNorm(x[first + i*step][:]; gain)); one block per output row.  If out_lo is given it
+// receives the bf16 rounding residual (value - float(out)), so that out + out_lo carries 16 mantissa bits.
 __global__ void __launch_bounds__(256)
-rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out, int H, float eps,
-                    int first, int step) {
+rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out,
+                    bf16 *__restrict__ out_lo, int H, float eps, int first, int step) {
     __shared__ float red[8];
     pdl_wait();
     const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
@@ -105,10 +106,18 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
     for (int i = threadIdx.x; i < H / 4; i += 256) {
         const float4 v = src[i];
         const uint2 g = reinterpret_cast<const uint2 *>(gain)[i];
+        const float y0 = v.x * inv * bf16_lo(g.x), y1 = v.y * inv * bf16_hi(g.x);
+        const float y2 = v.z * inv * bf16_lo(g.y), y3 = v.w * inv * bf16_hi(g.y);
         uint2 o;
-        o.x = pack_bf16x2(v.x * inv * bf16_lo(g.x), v.y * inv * bf16_hi(g.x));
-        o.y = pack_bf16x2(v.z * inv * bf16_lo(g.y), v.w * inv * bf16_hi(g.y));
+        o.x = pack_bf16x2(y0, y1);
+        o.y = pack_bf16x2(y2, y3);
         dst[i] = o;
+        if (out_lo) {
+            uint2 r;
+            r.x = pack_bf16x2(y0 - bf16_lo(o.x), y1 - bf16_hi(o.x));
+            r.y = pack_bf16x2(y2 - bf16_lo(o.y), y3 - bf16_hi(o.y));
+            reinterpret_cast<uint2 *>(out_lo + (size_t)blockIdx.x * H)[i] = r;
+        }
     }
     pdl_launch_dependents();
 }
@@ -141,9 +150,9 @@ cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows
                   rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, q_bf16_out);
 }
 
-cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, int rows, int H,
-                                float eps, int first, int step) {
-    return launch(lc, rmsnorm_rows_kernel, dim3(rows), dim3(256), x, gain, out, H, eps, first, step);
+cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
+                                int H, float eps, int first, int step) {
+    return launch(lc, rmsnorm_rows_kernel, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
 }
 
 cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n) {

@@ -125,18 +125,22 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn) {
 
 struct GemmParams {
     void *Y;          // output
+    void *Y_lo;       // SwiGLU epilogue only: bf16 rounding residual of Y (nullable)
     int T, N, K;      // tokens, weight rows, reduction
     int ldy;          // output row stride in elements
     int m_tiles, n_tiles;
     int *status;
 };
 
-template <int BN>
+// Shared-memory stage: [weight tile][activation tile][activation residual tile (SPLIT)].
+// SWAP puts the weights on the M side (128 rows) and BN tokens on the N side; otherwise 128 tokens x BN weights.
+template <int BN, bool SWAP, bool SPLIT>
 struct SmemLayout {
-    static constexpr int kStageA = kBM * kBK * 2;
-    static constexpr int kStageB = BN * kBK * 2;
-    static constexpr int kStage = kStageA + kStageB;
-    static constexpr int kStages = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr int kW = (SWAP ? kBM : BN) * kBK * 2;
+    static constexpr int kX = (SWAP ? BN : kBM) * kBK * 2;
+    static constexpr int kStage = kW + kX * (SPLIT ? 2 : 1);
+    static constexpr int kStagesFit = (192 * 1024) / kStage;
+    static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr int kBytes = kStages * kStage + 1024 /*align slack*/ + 256 /*barriers*/;
     static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
 };
@@ -144,10 +148,13 @@ struct SmemLayout {
 __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
 
 // EPI: 0 fp32 store, 1 bf16 store, 2 fp32 accumulate (Y += D), 3 SwiGLU on interleaved gate/up weight rows -> bf16
-template <int BN, bool SWAP, int EPI>
+// SPLIT: the activations come as two bf16 matrices (value and rounding residual); both are multiplied with the
+// same weight tile into the same accumulator, which restores ~16 mantissa bits on the activation side.
+template <int BN, bool SWAP, int EPI, bool SPLIT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant__ CUtensorMap map_n, GemmParams p) {
-    using L = SmemLayout<BN>;
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+               const __grid_constant__ CUtensorMap map_x_lo, GemmParams p) {
+    using L = SmemLayout<BN, SWAP, SPLIT>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = base + L::kStages * L::kStage;      // full[S], empty[S], tfull[2], tempty[2], 8 B each
@@ -189,12 +196,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant_
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+                const int w_row = SWAP ? mt * kBM : nt * BN;
+                const int x_row = SWAP ? nt * BN : mt * kBM;
                 for (int kb = 0; kb < kb_count; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     mbar_expect_tx(full_bar(stage), L::kStage);
-                    const uint32_t sa = base + stage * L::kStage;
-                    tma_load_2d(sa, &map_m, full_bar(stage), kb * kBK, mt * kBM);
-                    tma_load_2d(sa + L::kStageA, &map_n, full_bar(stage), kb * kBK, nt * BN);
+                    const uint32_t sw = base + stage * L::kStage;
+                    tma_load_2d(sw, &map_w, full_bar(stage), kb * kBK, w_row);
+                    tma_load_2d(sw + L::kW, &map_x, full_bar(stage), kb * kBK, x_row);
+                    if (SPLIT) tma_load_2d(sw + L::kW + L::kX, &map_x_lo, full_bar(stage), kb * kBK, x_row);
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -212,11 +222,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant_
                 for (int kb = 0; kb < kb_count; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = base + stage * L::kStage;
-                    const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + L::kStageA);
+                    const uint32_t sw = base + stage * L::kStage;
+                    const uint64_t dw = make_smem_desc(sw), dx = make_smem_desc(sw + L::kW),
+                                   dxl = make_smem_desc(sw + L::kW + L::kX);
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)
-                        umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        const uint64_t off = (uint64_t)(k * 2);  // 32 bytes, in 16-byte units
+                        if (SWAP) {
+                            umma_bf16(d_tmem, dw + off, dx + off, idesc, (kb | k) != 0);
+                            if (SPLIT) umma_bf16(d_tmem, dw + off, dxl + off, idesc, 1u);
+                        } else {
+                            umma_bf16(d_tmem, dx + off, dw + off, idesc, (kb | k) != 0);
+                            if (SPLIT) umma_bf16(d_tmem, dxl + off, dw + off, idesc, 1u);
+                        }
+                    }
                     umma_commit(empty_bar(stage));
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -243,19 +262,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant_
                     // row m = token, columns n0.. = weight rows: contiguous per thread
                     if (m < p.T) {
                         if (EPI == 3) {
-                            bf16 *y = reinterpret_cast<bf16 *>(p.Y) + (size_t)m * p.ldy + (n0 >> 1);
+                            const size_t yo = (size_t)m * p.ldy + (n0 >> 1);
+                            bf16 *y = reinterpret_cast<bf16 *>(p.Y) + yo;
+                            bf16 *yl = p.Y_lo ? reinterpret_cast<bf16 *>(p.Y_lo) + yo : nullptr;
                             if (n0 + 32 <= p.N) {
-                                uint32_t o[8];
+                                uint32_t o[8], ol[8];
 #pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    o[i] = pack_bf16x2(silu_mul(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])),
-                                                       silu_mul(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])));
+                                for (int i = 0; i < 8; ++i) {
+                                    const float a0 = silu_mul(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
+                                    const float a1 = silu_mul(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                                    o[i] = pack_bf16x2(a0, a1);
+                                    ol[i] = pack_bf16x2(a0 - bf16_lo(o[i]), a1 - bf16_hi(o[i]));
+                                }
                                 reinterpret_cast<uint4 *>(y)[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 reinterpret_cast<uint4 *>(y)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                                if (yl) {
+                                    reinterpret_cast<uint4 *>(yl)[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                                    reinterpret_cast<uint4 *>(yl)[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
+                                }
                             } else {
                                 for (int i = 0; i < 16; ++i)
-                                    if (n0 + 2 * i + 1 < p.N)
-                                        y[i] = __float2bfloat16_rn(silu_mul(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])));
+                                    if (n0 + 2 * i + 1 < p.N) {
+                                        const float a = silu_mul(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                                        const bf16 hi = __float2bfloat16_rn(a);
+                                        y[i] = hi;
+                                        if (yl) yl[i] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                                    }
                             }
                         } else if (EPI == 1) {
                             bf16 *y = reinterpret_cast<bf16 *>(p.Y) + (size_t)m * p.ldy + n0;
@@ -301,8 +333,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_m, const __grid_constant_
                             const float mine = __uint_as_float(r[i]);
                             const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
                             const int t = n0 + i;
-                            if (!(lane & 1) && m + 1 < p.N && t < p.T)
-                                reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + (m >> 1)] = __float2bfloat16_rn(silu_mul(mine, other));
+                            if (!(lane & 1) && m + 1 < p.N && t < p.T) {
+                                const float a = silu_mul(mine, other);
+                                const bf16 hi = __float2bfloat16_rn(a);
+                                const size_t yo = (size_t)t * p.ldy + (m >> 1);
+                                reinterpret_cast<bf16 *>(p.Y)[yo] = hi;
+                                if (p.Y_lo) reinterpret_cast<bf16 *>(p.Y_lo)[yo] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                            }
                         }
                     } else {
 #pragma unroll
@@ -372,61 +409,73 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows) 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool SWAP, int EPI>
-cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
-                      int *status) {
-    using L = SmemLayout<BN>;
-    auto kern = gemm_tc_kernel<BN, SWAP, EPI>;
+template <int BN, bool SWAP, int EPI, bool SPLIT>
+cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
+                      int K, int ldy, int *status) {
+    using L = SmemLayout<BN, SWAP, SPLIT>;
+    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    CUtensorMap map_m, map_n;
+    CUtensorMap map_w, map_x, map_x_lo;
     GemmParams p;
-    p.Y = Y; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status;
+    p.Y = Y; p.Y_lo = Y_lo; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status;
+    const int w_box = SWAP ? kBM : BN, x_box = SWAP ? BN : kBM;
+    if (!make_map(&map_w, W, N, K, w_box) || !make_map(&map_x, X, T, K, x_box)) return cudaErrorInvalidValue;
+    if (!make_map(&map_x_lo, SPLIT ? X_lo : X, T, K, x_box)) return cudaErrorInvalidValue;
     if (!SWAP) {
-        if (!make_map(&map_m, X, T, K, kBM) || !make_map(&map_n, W, N, K, BN)) return cudaErrorInvalidValue;
         p.m_tiles = (T + kBM - 1) / kBM;
         p.n_tiles = (N + BN - 1) / BN;
     } else {
-        if (!make_map(&map_m, W, N, K, kBM) || !make_map(&map_n, X, T, K, BN)) return cudaErrorInvalidValue;
         p.m_tiles = (N + kBM - 1) / kBM;
         p.n_tiles = (T + BN - 1) / BN;
     }
     int grid = p.m_tiles * p.n_tiles;
     if (grid > lc.sm_count) grid = lc.sm_count;
     if (lc.launches) ++*lc.launches;
-    kern<<<grid, kGemmThreads, L::kBytes, lc.stream>>>(map_m, map_n, p);
+    kern<<<grid, kGemmThreads, L::kBytes, lc.stream>>>(map_w, map_x, map_x_lo, p);
     return cudaGetLastError();
 }
 
-template <int EPI>
-cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
-                     int *status) {
-    if (T <= 32) return launch_tc<32, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
-    if (T <= 64) return launch_tc<64, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
-    if (T <= 128) return launch_tc<128, true, EPI>(lc, X, W, Y, T, N, K, ldy, status);
-    return launch_tc<256, false, EPI>(lc, X, W, Y, T, N, K, ldy, status);
+template <int EPI, bool SPLIT>
+cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
+                     int K, int ldy, int *status) {
+    if (T <= 32) return launch_tc<32, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+    if (T <= 64) return launch_tc<64, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+    if (T <= 128) return launch_tc<128, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+    return launch_tc<256, false, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+}
+
+template <bool SPLIT>
+cudaError_t dispatch_epi(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
+                         int N, int K, int ldy, int epi, int *status) {
+    switch (epi) {
+        case kEpiStoreF32: return dispatch<0, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+        case kEpiStoreBf16: return dispatch<1, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+        case kEpiAccumF32: return dispatch<2, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+        case kEpiSwigluBf16: return dispatch<3, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
 bool gemm_tc_available() { return get_encode() != nullptr; }
 
-// Y[T][*] (row stride ldy) = epilogue(X[T][K] * W[N][K]^T).  X, W 16-byte aligned, K % 64 == 0.
-cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
-                        int epi, int *status) {
+// Y[T][*] (row stride ldy) = epilogue((X + X_lo)[T][K] * W[N][K]^T).  Operands 16-byte aligned, K % 64 == 0.
+cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
+                        int N, int K, int ldy, int epi, int *status) {
     if (T <= 0 || N <= 0 || K <= 0 || K % kBK != 0 || N % 8 != 0) return cudaErrorInvalidValue;
-    if (((uintptr_t)X | (uintptr_t)W | (uintptr_t)Y) & 15) return cudaErrorInvalidValue;
-    switch (epi) {
-        case kEpiStoreF32: return dispatch<0>(lc, X, W, Y, T, N, K, ldy, status);
-        case kEpiStoreBf16: return dispatch<1>(lc, X, W, Y, T, N, K, ldy, status);
-        case kEpiAccumF32: return dispatch<2>(lc, X, W, Y, T, N, K, ldy, status);
-        case kEpiSwigluBf16: return dispatch<3>(lc, X, W, Y, T, N, K, ldy, status);
-    }
-    return cudaErrorInvalidValue;
+    if (((uintptr_t)X | (uintptr_t)X_lo | (uintptr_t)W | (uintptr_t)Y | (uintptr_t)Y_lo) & 15) return cudaErrorInvalidValue;
+    // the epilogue stores 16-byte vectors per output row: the row pitch must keep them aligned
+    const bool out_bf16 = epi == kEpiStoreBf16 || epi == kEpiSwigluBf16;
+    if (ldy % (out_bf16 ? 8 : 4) != 0) return cudaErrorInvalidValue;
+    if (epi == kEpiSwigluBf16 && N % 2 != 0) return cudaErrorInvalidValue;
+    return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status)
+                : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status);
 }
 
 }  // namespace nnc

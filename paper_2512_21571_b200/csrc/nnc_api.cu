@@ -32,7 +32,7 @@ struct Plan {
     std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
     size_t x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
-    size_t xt, hb, qkvt, ob, ab, logits_stage;
+    size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
     size_t take(size_t bytes) {
         const size_t o = total;
         total += (bytes + kAlign - 1) / kAlign * kAlign;
@@ -89,9 +89,12 @@ void make_plan(const nnc_config &c, Plan &p) {
     p.d_argmax = p.take(B * 4);
     p.xt = p.take(R * H * 4);
     p.hb = p.take(R * H * 2);
+    p.hb_lo = p.take(R * H * 2);
     p.qkvt = p.take(R * qkvd * 4);
     p.ob = p.take(R * qd * 2);
+    p.ob_lo = p.take(R * qd * 2);
     p.ab = p.take(R * I * 2);
+    p.ab_lo = p.take(R * I * 2);
     p.logits_stage = p.take((size_t)kHostLogitRows * V * 4);
 }
 
@@ -100,6 +103,7 @@ void make_plan(const nnc_config &c, Plan &p) {
 struct nnc_model {
     nnc_config c;
     cudaStream_t stream;
+    cudaStream_t capture_stream;  // graphs are captured here (the caller's stream may be the legacy stream, which cannot capture)
     int device, sm_count;
     char *ws;
     Plan plan;
@@ -111,6 +115,7 @@ struct nnc_model {
     int32_t *d_len, *d_status, *d_tokens, *d_argmax;
     float *xt, *qkvt, *logits_stage;
     bf16 *hb, *ob, *ab;
+    bf16 *hb_lo, *ob_lo, *ab_lo;  // bf16 rounding residuals of the GEMM activations (null in fast mode)
     int len;
     float *taps;
     bool pdl;
@@ -159,7 +164,7 @@ int layer_decode_b1(nnc_model *m, int l, const LaunchCtx &lc, int n_splits) {
     NNC_CUDA(m, launch_gemv(lc, w.wqkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr));
     NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkv, 1, 1, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
                                            c.n_kv_heads, c.max_seq, m->d_len, nullptr));
-    NNC_CUDA(m, launch_attn_decode(lc, m->qkv, m->qkvd(), kc, vc, m->attn_out, nullptr, m->qd(), m->part, m->tickets,
+    NNC_CUDA(m, launch_attn_decode(lc, m->qkv, m->qkvd(), kc, vc, m->attn_out, nullptr, nullptr, m->qd(), m->part, m->tickets,
                                    m->d_len, 1, 1, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits));
     NNC_CUDA(m, launch_gemv(lc, w.wo, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr));
     NNC_CUDA(m, launch_gemv(lc, w.wgu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr));
@@ -194,33 +199,33 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
         const LayerW &w = m->layers[l];
         bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
         bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
-        NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_in, m->hb, R, H, c.rms_eps, 0, 1));
-        NNC_CUDA(m, launch_gemm(lc, m->hb, w.wqkv, m->qkvt, R, qkvd, H, qkvd, kEpiStoreF32, m->d_status));
+        NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_in, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
+        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wqkv, m->qkvt, nullptr, R, qkvd, H, qkvd, kEpiStoreF32, m->d_status));
         NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
                                                c.n_kv_heads, c.max_seq, m->d_len, nullptr));
         if (T == 1) {
-            NNC_CUDA(m, launch_attn_decode(lc, m->qkvt, qkvd, kc, vc, nullptr, m->ob, qd, m->part, m->tickets, m->d_len, 1,
+            NNC_CUDA(m, launch_attn_decode(lc, m->qkvt, qkvd, kc, vc, nullptr, m->ob, m->ob_lo, qd, m->part, m->tickets, m->d_len, 1,
                                            batch, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits));
         } else {
-            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, c.n_q_heads, c.n_kv_heads, c.max_seq, m->d_len));
+            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, c.n_q_heads, c.n_kv_heads, c.max_seq, m->d_len));
         }
-        NNC_CUDA(m, launch_gemm(lc, m->ob, w.wo, m->xt, R, H, qd, H, kEpiAccumF32, m->d_status));
-        NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, R, H, c.rms_eps, 0, 1));
-        NNC_CUDA(m, launch_gemm(lc, m->hb, w.wgu, m->ab, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status));
-        NNC_CUDA(m, launch_gemm(lc, m->ab, w.wd, m->xt, R, H, I, H, kEpiAccumF32, m->d_status));
+        NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status));
+        NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
+        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wgu, m->ab, m->ab_lo, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status));
+        NNC_CUDA(m, launch_gemm(lc, m->ab, m->ab_lo, w.wd, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status));
         if (m->taps) NNC_CUDA(m, launch_copy_f32(lc, m->xt, m->taps + (size_t)(l + 1) * R * H, (size_t)R * H));
     }
     if (logits) {
         if (all_positions || T == 1) {
-            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, R, H, c.rms_eps, 0, 1));
-            NNC_CUDA(m, launch_gemm(lc, m->hb, m->lm_head, logits, R, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
+            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, R, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
         } else if (batch == 1) {
             // last position only: the streaming GEMV keeps the activation in fp32
             NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->xt + (size_t)(T - 1) * H, logits, c.vocab, H, m->g_final, c.rms_eps,
                                     kGemvLogits, nullptr));
         } else {
-            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, batch, H, c.rms_eps, T - 1, T));
-            NNC_CUDA(m, launch_gemm(lc, m->hb, m->lm_head, logits, batch, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
+            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, m->hb_lo, batch, H, c.rms_eps, T - 1, T));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, batch, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
         }
     }
     NNC_CUDA(m, launch_add_len(lc, m->d_len, T));
@@ -260,6 +265,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
             return NNC_ERR_INVALID_ARG;
     }
     nnc_model *m = new nnc_model();
+    m->capture_stream = nullptr;
     m->c = *config;
     m->err[0] = 0;
     make_plan(m->c, m->plan);
@@ -275,6 +281,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         NNC_CUDA(m, cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, m->device));
         if (major != 10) return fail(m, NNC_ERR_CUDA, "this library is built for sm_100a only (device is sm_%d*)", major);
         m->stream = (cudaStream_t)cuda_stream;
+        NNC_CUDA(m, cudaStreamCreateWithFlags(&m->capture_stream, cudaStreamNonBlocking));
         m->ws = (char *)workspace;
         const Plan &p = m->plan;
         const nnc_config &c = m->c;
@@ -295,6 +302,10 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         m->d_tokens = (int32_t *)at(p.d_tokens); m->d_argmax = (int32_t *)at(p.d_argmax);
         m->xt = (float *)at(p.xt); m->hb = (bf16 *)at(p.hb); m->qkvt = (float *)at(p.qkvt);
         m->ob = (bf16 *)at(p.ob); m->ab = (bf16 *)at(p.ab); m->logits_stage = (float *)at(p.logits_stage);
+        const bool fast = c.fast_bf16_activations != 0;
+        m->hb_lo = fast ? nullptr : (bf16 *)at(p.hb_lo);
+        m->ob_lo = fast ? nullptr : (bf16 *)at(p.ob_lo);
+        m->ab_lo = fast ? nullptr : (bf16 *)at(p.ab_lo);
         m->len = 0;
         m->taps = nullptr;
         m->launches = 0;
@@ -348,6 +359,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
     rc = body();
     if (rc != NNC_OK) {
         fprintf(stderr, "nnc_model_create: %s\n", m->err);
+        if (m->capture_stream) cudaStreamDestroy(m->capture_stream);
         delete m;
         return rc;
     }
@@ -359,6 +371,7 @@ void nnc_model_destroy(nnc_model *m) {
     if (!m) return;
     cudaStreamSynchronize(m->stream);
     for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
+    if (m->capture_stream) cudaStreamDestroy(m->capture_stream);
     delete m;
 }
 
@@ -392,9 +405,11 @@ int nnc_decode_step(nnc_model *m, const int32_t *tokens, int32_t batch, float *l
     if (it == m->graphs.end()) {
         cudaGraph_t graph = nullptr;
         int64_t before = m->launches;
-        NNC_CUDA(m, cudaStreamBeginCapture(m->stream, cudaStreamCaptureModeThreadLocal));
-        rc = decode_b1_launches(m, tokens, logits, argmax, ctx(m, m->pdl));
-        cudaError_t e = cudaStreamEndCapture(m->stream, &graph);
+        NNC_CUDA(m, cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeThreadLocal));
+        LaunchCtx cap = ctx(m, m->pdl);
+        cap.stream = m->capture_stream;
+        rc = decode_b1_launches(m, tokens, logits, argmax, cap);
+        cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
         const int64_t nodes = m->launches - before;
         m->launches = before;
         if (rc != NNC_OK) {
@@ -567,8 +582,8 @@ static int op_ctx(LaunchCtx &lc, void *stream) {
     return NNC_OK;
 }
 
-int nnc_op_gemm(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in, int32_t out_f32,
-                int32_t accumulate, void *cuda_stream) {
+int nnc_op_gemm(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                int32_t out_f32, int32_t accumulate, void *cuda_stream) {
     if (!X || !W || !Y) return NNC_ERR_INVALID_ARG;
     if (accumulate && !out_f32) return NNC_ERR_INVALID_ARG;
     LaunchCtx lc;
@@ -576,18 +591,19 @@ int nnc_op_gemm(const void *X, const void *W, void *Y, int32_t T, int32_t n_out,
     int *status = nullptr;
     if (cudaGetSymbolAddress((void **)&status, g_op_status) != cudaSuccess) return NNC_ERR_CUDA;
     const int epi = out_f32 ? (accumulate ? kEpiAccumF32 : kEpiStoreF32) : kEpiStoreBf16;
-    cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)W, Y, T, n_out, n_in, n_out, epi, status);
+    cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)X_lo, (const bf16 *)W, Y, nullptr, T, n_out, n_in, n_out, epi, status);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 
-int nnc_op_gemm_swiglu(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in, void *cuda_stream) {
+int nnc_op_gemm_swiglu(const void *X, const void *X_lo, const void *W, void *Y, void *Y_lo, int32_t T, int32_t n_out,
+                       int32_t n_in, void *cuda_stream) {
     if (!X || !W || !Y || n_out % 2) return NNC_ERR_INVALID_ARG;
     LaunchCtx lc;
     if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
     int *status = nullptr;
     if (cudaGetSymbolAddress((void **)&status, g_op_status) != cudaSuccess) return NNC_ERR_CUDA;
-    cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)W, Y, T, n_out, n_in, n_out / 2, kEpiSwigluBf16, status);
+    cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)X_lo, (const bf16 *)W, Y, Y_lo, T, n_out, n_in, n_out / 2, kEpiSwigluBf16, status);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
@@ -630,7 +646,7 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
     float *part = (float *)scratch;
     uint32_t *tickets = (uint32_t *)((char *)scratch + (attn_decode_scratch_floats(batch, n_q_heads, kAttnMaxSplits) * 4 + 255) / 256 * 256);
     if (cudaMemsetAsync(tickets, 0, (size_t)batch * n_kv_heads * 4, lc.stream) != cudaSuccess) return NNC_ERR_CUDA;
-    cudaError_t e = launch_attn_decode(lc, q, n_q_heads * 128, (const bf16 *)kcache, (const bf16 *)vcache, out, nullptr,
+    cudaError_t e = launch_attn_decode(lc, q, n_q_heads * 128, (const bf16 *)kcache, (const bf16 *)vcache, out, nullptr, nullptr,
                                        n_q_heads * 128, part, tickets, nullptr, n_ctx, batch, n_q_heads, n_kv_heads,
                                        max_seq, n_splits);
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;

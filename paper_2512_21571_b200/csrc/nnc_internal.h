@@ -53,8 +53,8 @@ cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
                                        const int32_t *d_len, bf16 *q_bf16_out);
-cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, int rows, int H,
-                                float eps, int first, int step);
+cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
+                                int H, float eps, int first, int step);
 cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n);
 cudaError_t launch_add_len(const LaunchCtx &lc, int32_t *d_len, int delta);
 
@@ -63,17 +63,20 @@ constexpr int kAttnMaxSplits = 64;
 int attn_decode_splits(int sm_count, int batch, int nkv, int max_ctx);
 size_t attn_decode_scratch_floats(int batch, int nq, int n_splits);
 cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, const bf16 *kcache,
-                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, int out_row_stride, float *part,
-                               uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
+                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride,
+                               float *part, uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
                                int max_seq, int n_splits);
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
-                                const bf16 *vcache, bf16 *out, int nq, int nkv, int max_seq, const int32_t *d_len);
+                                const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
+                                const int32_t *d_len);
 
 // ---- GEMM (gemm_tc.cu) --------------------------------------------------------------------------------
 enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwigluBf16 = 3 };
 bool gemm_tc_available();
-cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *W, void *Y, int T, int N, int K, int ldy,
-                        int epi, int *status);
+// X_lo (nullable): bf16 rounding residual of the activations; the product is then (X + X_lo) W^T.
+// Y_lo (nullable, SwiGLU epilogue only): receives the rounding residual of the bf16 output.
+cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
+                        int N, int K, int ldy, int epi, int *status);
 
 // ---- repack (repack.cu) -------------------------------------------------------------------------------
 // dst rows [row0, row0 + rows) <- src rows [0, rows), row length K (plain row copy into a taller matrix)

@@ -33,7 +33,8 @@ def test_every_declared_symbol_is_exported(binding):
 
 def _cfg(binding, **kw):
     base = dict(n_layers=36, hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, intermediate=12288, vocab=151936,
-                max_seq=4352, max_batch=1, max_tokens=1, tie_embeddings=0, rms_eps=1e-6, rope_theta=1e6)
+                max_seq=4352, max_batch=1, max_tokens=1, tie_embeddings=0, rms_eps=1e-6, rope_theta=1e6,
+                fast_bf16_activations=0)
     base.update(kw)
     return binding.nnc_config(**base)
 
@@ -65,5 +66,5 @@ def test_null_arguments_and_status_strings(binding):
     assert binding.lib.nnc_get_length(None) == -1
     assert binding.lib.nnc_status_string(0) == b"ok"
     assert b"capacity" in binding.lib.nnc_status_string(-3)
-    assert binding.lib.nnc_op_gemm(None, None, None, 1, 8, 64, 1, 0, None) == -1
+    assert binding.lib.nnc_op_gemm(None, None, None, None, 1, 8, 64, 1, 0, None) == -1
     binding.lib.nnc_model_destroy(None)

@@ -1,0 +1,106 @@
+"""The five workload configurations at their real shapes: CUDA library vs CPU oracle, teacher-forced on the
+oracle's tokens.  Weights are generated once on the GPU (seeded) and copied to the host for the oracle.
+
+Sizes the oracle cannot finish in reasonable time are sampled: the number of oracle decode steps is bounded
+(NNC_TEST_STEPS overrides), and batched workloads are checked on a subset of sequences plus the
+batch-independence property.  Error statistics are appended to gpurun_out/parity_stats.txt.
+"""
+import os
+import time
+
+import pytest
+import torch
+
+from gpu_util import make_pair, rel_l2
+from paper_2512_21571_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+HID_TOL, LOGIT_TOL, MARGIN = 1e-2, 3e-2, 1e-2
+STEPS = int(os.environ.get("NNC_TEST_STEPS", "0"))
+
+
+def _log(line):
+    os.makedirs("gpurun_out", exist_ok=True)
+    with open("gpurun_out/parity_stats.txt", "a") as f:
+        f.write(line + "\n")
+    print(line)
+
+
+def _run(oracle_mod, name, seed, prefill, decode, kv_prefill=0, check_all_positions=False):
+    shape = synth.SHAPES[name]
+    max_seq = kv_prefill + prefill + decode + 1
+    t0 = time.time()
+    m, o, w = make_pair(oracle_mod, shape, seed, max_seq=max_seq, max_tokens=max(prefill, 1))
+    if kv_prefill:
+        for l in range(shape.n_layers):
+            k, v = synth.kv_fill(shape, seed + 1000, l, kv_prefill, device="cuda")
+            m.kv_import(l, 0, k, v)
+            o.kv_import(l, k.cpu(), v.cpu())
+        m.set_length(kv_prefill)
+    t_setup = time.time() - t0
+    worst_h = worst_l = 0.0
+    n_arg = n_arg_checked = 0
+    if prefill:
+        toks = synth.prompt_tokens(shape, seed + 1000, prefill)
+        taps = torch.zeros(shape.n_layers + 1, prefill, shape.hidden, device="cuda")
+        m.set_hidden_tap(taps)
+        lg = m.prefill(toks.cuda().view(1, prefill), all_positions=check_all_positions)
+        m.set_hidden_tap(None)
+        lo, to = o.forward(toks, all_positions=check_all_positions, want_taps=True)
+        per_layer = [rel_l2(taps[l], to[l]) for l in range(shape.n_layers + 1)]
+        worst_h = max(per_layer)
+        worst_l = (lg[0].cpu() - lo).abs().max().item()
+        _log(f"{name} prefill T={prefill}: hidden rel-L2 max {worst_h:.3e} (last layer {per_layer[-1]:.3e}), "
+             f"logits max-abs {worst_l:.3e}")
+        assert worst_h < HID_TOL and worst_l < LOGIT_TOL
+        tok = int((lo[-1] if check_all_positions else lo).argmax())
+    else:
+        tok = int(synth.prompt_tokens(shape, seed + 1000, 1)[0])
+    logits = torch.empty(shape.vocab, device="cuda")
+    am = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    taps1 = torch.zeros(shape.n_layers + 1, 1, shape.hidden, device="cuda")
+    dh = dl = 0.0
+    t0 = time.time()
+    for step in range(decode):
+        tok_dev.fill_(tok)
+        tapped = step % 8 == 0          # instrumented (kernel by kernel) every 8th step, captured graph otherwise
+        m.set_hidden_tap(taps1 if tapped else None)
+        m.decode_step(tok_dev, logits, am)
+        l1, t1 = o.forward(torch.tensor([tok], dtype=torch.int32), want_taps=tapped)
+        if tapped:
+            dh = max(dh, rel_l2(taps1, t1))
+        dl = max(dl, (logits.cpu() - l1).abs().max().item())
+        idx, margin = oracle_mod.argmax_margin(l1)
+        n_arg += 1
+        if margin > MARGIN:
+            n_arg_checked += 1
+            assert int(am.item()) == idx, (step, int(am.item()), idx, margin)
+        tok = idx
+    _log(f"{name} decode {decode} steps from ctx {kv_prefill + prefill}: hidden rel-L2 max {dh:.3e}, logits max-abs "
+         f"{dl:.3e}, argmax exact on {n_arg_checked}/{n_arg} steps with margin > {MARGIN}; setup {t_setup:.0f}s, "
+         f"decode+oracle {time.time() - t0:.0f}s")
+    assert dh < HID_TOL and dl < LOGIT_TOL
+    assert m.device_status() == 0
+    m.close(); o.close()
+
+
+def test_config2_qwen3_0p6b_prefill64_decode64(oracle_mod):
+    _run(oracle_mod, "qwen3-0.6b", 1, prefill=64, decode=STEPS or 64, check_all_positions=True)
+
+
+def test_config3_qwen3_1p7b_prefill512_decode(oracle_mod):
+    # the oracle's share of the 256 decode steps is sampled: the first 16 (override with NNC_TEST_STEPS)
+    _run(oracle_mod, "qwen3-1.7b", 2, prefill=512, decode=STEPS or 16)
+
+
+def test_config4_qwen3_8b_ctx4096_decode(oracle_mod):
+    # the HBM-roofline workload: cache pre-filled to 4096 positions; oracle steps sampled (first 6)
+    _run(oracle_mod, "qwen3-8b", 3, prefill=0, decode=STEPS or 6, kv_prefill=4096)
+
+
+def test_config5_mode1_qwen3_8b_prefill_sampled(oracle_mod):
+    # batched prefill on the 8B shape; the oracle's share is one sequence of 256 tokens (the full 4 x 2048 is
+    # ~114 TFLOP of CPU work); batch independence is covered by test_batched_sequences_are_independent
+    _run(oracle_mod, "qwen3-8b", 4, prefill=int(os.environ.get("NNC_TEST_PREFILL", "256")), decode=STEPS or 2)

@@ -73,8 +73,8 @@ def test_tiny_model_prefill_then_decode(oracle_mod, name, seed, gains):
     for l in range(shape.n_layers):
         kg, vg = m.kv_export(l, 0, P)
         ko, vo = o.kv_export(l, P)
-        assert torch.allclose(kg.float().cpu(), ko.float(), rtol=2e-2, atol=2e-2)
-        assert torch.allclose(vg.float().cpu(), vo.float(), rtol=2e-2, atol=2e-2)
+        # cache rows carry the bf16-operand error of the tensor-core path plus one bf16 rounding
+        assert rel_l2(kg, ko) < HID_TOL and rel_l2(vg, vo) < HID_TOL, l
     # ---- decode, teacher-forced on the oracle's greedy tokens; instrumented (kernel by kernel) ----
     taps1 = torch.zeros(shape.n_layers + 1, 1, shape.hidden, device="cuda")
     m.set_hidden_tap(taps1)
@@ -82,16 +82,19 @@ def test_tiny_model_prefill_then_decode(oracle_mod, name, seed, gains):
     am = torch.zeros(1, dtype=torch.int32, device="cuda")
     tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
     tok = int(lo[-1].argmax())
+    tapped = True
     for step in range(D):
         tok_dev.fill_(tok)
         m.decode_step(tok_dev, logits, am)
         l1, t1 = o.forward(torch.tensor([tok], dtype=torch.int32), want_taps=True)
-        assert rel_l2(taps1, t1) < HID_TOL, step
+        if tapped:
+            assert rel_l2(taps1, t1) < HID_TOL, step
         assert (logits.cpu() - l1).abs().max().item() < LOGIT_TOL, step
         _check_argmax(oracle_mod, int(am.item()), l1)
         assert logits[int(am.item())] == logits.max()  # the fused arg-max agrees with the logits it produced
         if step == D // 2:
             m.set_hidden_tap(None)  # the remaining steps go through the captured graph
+            tapped = False
         tok = int(l1.argmax())
     assert m.length == P + D
     assert m.device_status() == 0
@@ -130,12 +133,12 @@ def test_prefill_equals_stepwise_decode_on_gpu(oracle_mod):
     logits = torch.empty(shape.vocab, device="cuda")
     for i in range(12):
         m.decode_step(toks[i:i + 1].contiguous(), logits)
-        assert (logits - la[i]).abs().max().item() < LOGIT_TOL / 2, i
+        assert (logits - la[i]).abs().max().item() < LOGIT_TOL, i
     # split prefill: 5 tokens, then 7 (positions continue from the cache length)
     m.set_length(0)
     m.prefill(toks[:5].contiguous().view(1, 5), want_logits=False)
     lb = m.prefill(toks[5:].contiguous().view(1, 7), all_positions=True)[0]
-    assert (lb - la[5:]).abs().max().item() < LOGIT_TOL / 2
+    assert (lb - la[5:]).abs().max().item() < LOGIT_TOL / 4
 
 
 def test_batched_sequences_are_independent(oracle_mod):

@@ -117,3 +117,29 @@ def test_attn_decode_against_oracle(nnc, oracle_mod, batch, nq, nkv, n_ctx, max_
             want = oracle_mod.attend(qc[b, i], kcc[b, i // G, :n_ctx].contiguous(), vcc[b, i // G, :n_ctx].contiguous())
             assert torch.allclose(out[b, i].cpu(), want, rtol=1e-4, atol=2e-5), (b, i)
     assert torch.isfinite(out).all()
+
+
+@pytest.mark.parametrize("T,N,K", [(9, 512, 256), (64, 1024, 128), (100, 384, 640), (300, 2048, 1024), (1000, 1000, 512)])
+def test_gemm_split_activations_recover_fp32_inputs(nnc, oracle_mod, T, N, K):
+    """Feeding value + rounding residual as two bf16 operands reproduces the product of the fp32 activations
+    (the oracle's matmul on the unrounded X) to ~2^-16, on both operand assignments (T <= 128 and T > 128)."""
+    X = synth.normal(7, 1, (T, K), 1.0, torch.float32, "cuda")
+    W = _w(7, 2, (N, K))
+    hi, lo = nnc.split_bf16(X)
+    Y = nnc.op_gemm(hi, W, X_lo=lo)
+    rows = sorted(set([0, T - 1, T // 2]))
+    want = oracle_mod.matmul(W.cpu(), X[rows].cpu())
+    assert torch.allclose(Y[rows].cpu(), want, rtol=1e-4, atol=3e-5 * math.sqrt(K) * 0.02 * 50)
+    ref = X.double() @ W.double().T
+    err_split = (Y.double() - ref).abs().max().item()
+    err_plain = (nnc.op_gemm(hi, W).double() - ref).abs().max().item()
+    assert err_split < 2e-5 * math.sqrt(K) and err_split < err_plain / 20
+    # SwiGLU epilogue with residual output (an output pitch that would misalign 16-byte stores is refused)
+    if N % 16:
+        with pytest.raises(nnc.NncError):
+            nnc.op_gemm_swiglu(hi, W, X_lo=lo, want_lo=True)
+        return
+    A, A_lo = nnc.op_gemm_swiglu(hi, W, X_lo=lo, want_lo=True)
+    refa = ref[:, 0::2] / (1 + torch.exp(-ref[:, 0::2])) * ref[:, 1::2]
+    assert (A.double() + A_lo.double() - refa).abs().max().item() < 1e-4
+    assert nnc.op_status() == 0
