@@ -189,6 +189,23 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
                        int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_ctx, void *scratch,
                        void *cuda_stream);
 
+/* The same operation for callers that cannot allocate device memory (the paper has no counterpart: this is a
+ * deployment convenience of this library).  A plug-in that is handed only its inputs and outputs, or a process
+ * whose device memory is owned by another runtime's pool, cannot produce the scratch buffer above; here the
+ * scratch lives in a fixed array inside the library image (NNC_ATTN_STATIC_SCRATCH_BYTES per GPU, held from
+ * library load until process exit) and the call allocates nothing.
+ *   - Needs above that size (nnc_attn_scratch_bytes(batch, n_q_heads, n_ctx) > NNC_ATTN_STATIC_SCRATCH_BYTES,
+ *     i.e. roughly batch * n_q_heads > 120) return NNC_ERR_CAPACITY, print one line to stderr, launch nothing.
+ *   - Every call on a device shares the array and finds the previous call's contents in it; the call clears
+ *     what must start at zero itself.  Calls that overlap on the GPU (two streams, two threads) race on the
+ *     array: serialise them.
+ *   - The first call on each device looks up the array's device address; issue that first call outside any
+ *     stream capture. */
+#define NNC_ATTN_STATIC_SCRATCH_BYTES (4u << 20)
+int nnc_op_attn_decode_static(const float *q, const void *kcache, const void *vcache, float *out, int32_t batch,
+                              int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_ctx,
+                              void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -69,6 +69,8 @@ EXPORTS = {
     "nnc_attn_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
     "nnc_op_attn_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "nnc_op_attn_decode_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                            C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
 }
 for _name, (_res, _args) in EXPORTS.items():
     _fn = getattr(lib, _name)
@@ -275,4 +277,16 @@ def op_attn_decode(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tensor, 
     _ok(lib.nnc_op_attn_decode(_dev(q, torch.float32), _dev(kcache, torch.bfloat16), _dev(vcache, torch.bfloat16),
                                out.data_ptr(), batch, nq, nkv, max_seq, n_ctx, scratch.data_ptr(), _stream_ptr()),
         "nnc_op_attn_decode")
+    return out
+
+
+def op_attn_decode_static(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tensor, n_ctx: int):
+    """nnc_op_attn_decode_static: as op_attn_decode, with the scratch in the library's built-in array (for callers
+    that cannot allocate).  The output tensor is the only buffer this wrapper creates."""
+    batch, nq, d = q.shape
+    _, nkv, max_seq, _ = kcache.shape
+    out = torch.empty_like(q)
+    _ok(lib.nnc_op_attn_decode_static(_dev(q, torch.float32), _dev(kcache, torch.bfloat16), _dev(vcache, torch.bfloat16),
+                                      out.data_ptr(), batch, nq, nkv, max_seq, n_ctx, _stream_ptr()),
+        "nnc_op_attn_decode_static")
     return out
