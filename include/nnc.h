@@ -176,7 +176,11 @@ int nnc_op_status(int32_t *status_out);
 
 /* y[n_out] = W[n_out][n_in] x (batch-1 streaming GEMV, fp32 accumulate).  x fp32 [n_in]; y fp32.
  * If gain != NULL (bf16 [n_in]) x is first RMS-normalised with that gain and eps.
- * mode 0: y = Wx;  mode 1: y += Wx (residual);  mode 2: rows interleaved gate/up, y[n_out/2] = silu(g)*u. */
+ * mode 0: y = Wx;  mode 1: y += Wx (residual);  mode 2: rows interleaved gate/up, y[n_out/2] = silu(g)*u.
+ * mode | NNC_GEMV_CHAINED: launch the way the decode step does, with programmatic stream serialization, so that
+ * back-to-back calls on one stream overlap the next kernel's weight prefetch with the previous kernel's tail
+ * (x and y of consecutive chained calls must then not depend on each other's weights buffer being rewritten). */
+#define NNC_GEMV_CHAINED 0x100
 int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t n_in, const void *gain,
                 float eps, int32_t mode, void *cuda_stream);
 

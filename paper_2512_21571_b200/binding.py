@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnnc.so")
+LIB_PATH = os.environ.get("NNC_LIBRARY") or os.path.join(_HERE, "libnnc.so")   # NNC_LIBRARY: another build of the same ABI
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_21571_b200.build` "
@@ -257,13 +257,17 @@ def op_status() -> int:
     return st.value
 
 
+GEMV_CHAINED = 0x100
+
+
 def op_gemv(W: torch.Tensor, x: torch.Tensor, mode: int = 0, gain: Optional[torch.Tensor] = None, eps: float = 1e-6,
-            y: Optional[torch.Tensor] = None):
+            y: Optional[torch.Tensor] = None, chained: bool = False):
     N, K = W.shape
     if y is None:
-        y = torch.empty(N // 2 if mode == 2 else N, dtype=torch.float32, device="cuda")
+        y = torch.empty(N // 2 if (mode & 0xff) == 2 else N, dtype=torch.float32, device="cuda")
     _ok(lib.nnc_op_gemv(_dev(W, torch.bfloat16), _dev(x, torch.float32), _dev(y, torch.float32), N, K,
-                        _dev(gain, torch.bfloat16) if gain is not None else None, eps, mode, _stream_ptr()), "nnc_op_gemv")
+                        _dev(gain, torch.bfloat16) if gain is not None else None, eps,
+                        mode | (GEMV_CHAINED if chained else 0), _stream_ptr()), "nnc_op_gemv")
     return y
 
 

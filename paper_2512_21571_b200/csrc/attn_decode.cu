@@ -1,13 +1,20 @@
-// GQA split-K flash-decode: one query token per sequence against a contiguous bf16 KV cache.
+// GQA split-K flash-decode: one query token per sequence against a contiguous bf16 KV cache, optionally fused
+// with the per-head QK-RMSNorm + RoPE of the new token and the append of its K/V row.
 //
-// Grid (n_splits, n_kv_heads, batch), 128 threads.  A CTA owns one KV head and one contiguous range of
-// positions; the G query heads that share the KV head ride along, so every K/V byte is loaded once and feeds
-// G dot products.  Positions are walked in tiles of 128 with an online softmax; 16 lanes cover one position
-// (16 bytes each), so a warp load is two fully used 256-byte cache rows.  Each CTA emits (m, l, o~) for its
-// range; the CTA that finishes last for a (sequence, KV head) folds the partials in split order (a ticket
-// counter, nobody waits), which keeps the result independent of arrival order.
-//
-// HBM-bound on K/V bytes; scores and probabilities never leave shared memory / registers.
+// HBM-bound on K/V bytes (2 * 2 * n_kv_heads * 128 bytes per cached position), so the kernel is arranged for
+// wide loads and few instructions per byte:
+//   - grid (n_splits, n_kv_heads, batch), 4 warps.  A CTA owns one KV head and one contiguous range of
+//     positions; its G query heads ride along, so every K/V byte is loaded once and feeds G dot products.
+//   - the two products run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 accumulate) with
+//     the G query heads as the (padded) 16-row operand.  Q and the probabilities are fed as two bf16 terms each
+//     (value + rounding residual), so the result keeps fp32-level accuracy.  K and V fragments are loaded
+//     straight from global memory as 16-byte vectors: the contraction index of Q.K^T (the head dimension) and the
+//     output column index of P.V are permuted so that what a thread needs is contiguous in the cache row.
+//   - every warp walks its own blocks of 16 positions with a private online softmax; warps, then CTAs, are
+//     merged through (m, l, o~) partials.  The CTA that finishes last for a (sequence, KV head) folds the
+//     partials in split order (a ticket counter; nobody waits), so the result does not depend on arrival order.
+//   - before waiting on the preceding kernel, the CTA asks for its K/V range to be brought into L2
+//     (cp.async.bulk.prefetch): the cache rows of earlier positions do not depend on that kernel.
 #include "common.cuh"
 #include "nnc_internal.h"
 
@@ -15,33 +22,101 @@ namespace nnc {
 
 namespace {
 
-constexpr int kTile = 128;
 constexpr int kPartStride = kHeadDim + 2;  // o~[128], m, l
+constexpr int kWarps = 4;
 
-__device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8]) {
-    f[0] = bf16_lo(u.x); f[1] = bf16_hi(u.x); f[2] = bf16_lo(u.y); f[3] = bf16_hi(u.y);
-    f[4] = bf16_lo(u.z); f[5] = bf16_hi(u.z); f[6] = bf16_lo(u.w); f[7] = bf16_hi(u.w);
+__device__ __forceinline__ uint4 ldg_cg(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 
-template <int G>
-__global__ void __launch_bounds__(128)
-attn_decode_kernel(const float *__restrict__ q, int q_row_stride, const bf16 *__restrict__ kcache,
-                   const bf16 *__restrict__ vcache, float *__restrict__ out_f32, bf16 *__restrict__ out_bf16,
-                   bf16 *__restrict__ out_bf16_lo, int out_row_stride, float *__restrict__ part, uint32_t *__restrict__ tickets,
-                   const int32_t *__restrict__ d_len, int len_add, int nkv, int max_seq, int n_splits) {
-    __shared__ float sc[G][kTile];       // scores, then probabilities, of the current tile
-    __shared__ float red[4][G][kHeadDim];
-    __shared__ float s_m[G], s_l[G], s_alpha[G];
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    // rows 8..15 of the 16-row operand are padding: a1 = a3 = 0
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+
+// value + residual bf16 pairs of two floats: hi holds bf16(x), lo holds bf16(x - hi)
+__device__ __forceinline__ void split2(float x, float y, uint32_t &hi, uint32_t &lo) {
+    hi = pack_bf16x2(x, y);
+    lo = pack_bf16x2(x - bf16_lo(hi), y - bf16_hi(hi));
+}
+
+struct AttnParams {
+    const float *q;          // [batch][q_row_stride]: query heads first; FUSED: then key heads, then value heads (raw)
+    int q_row_stride;
+    bf16 *kcache, *vcache;   // this layer: [batch][nkv][max_seq][128]
+    float *out_f32;          // [batch][out_row_stride] or null
+    bf16 *out_bf16, *out_bf16_lo;
+    int out_row_stride;
+    float *part;
+    uint32_t *tickets;
+    const int32_t *d_len;    // cached positions before this call (null = 0)
+    int len_add;             // positions attended = *d_len + len_add
+    int nkv, max_seq, n_splits;
+    const bf16 *g_q, *g_k;   // FUSED: per-head RMSNorm gains
+    const float *rope;       // FUSED: [max_seq][64][2]
+    float eps;
+};
+
+// RMSNorm over the 128 elements of one head + rotation by the table row; lane l owns elements 2l, 2l+1 and their
+// rotation partners 2l+64, 2l+65 (half-split pairing).
+__device__ __forceinline__ void norm_rope(float2 &a, float2 &b, const bf16 *gain, const float *rope_row, float eps, int lane) {
+    const float ss = warp_sum(a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y);
+    const float inv = rsqrtf(ss * (1.f / kHeadDim) + eps);
+    const uint32_t ga = reinterpret_cast<const uint32_t *>(gain)[lane];
+    const uint32_t gb = reinterpret_cast<const uint32_t *>(gain + 64)[lane];
+    a.x *= inv * bf16_lo(ga); a.y *= inv * bf16_hi(ga);
+    b.x *= inv * bf16_lo(gb); b.y *= inv * bf16_hi(gb);
+    const float4 cs = reinterpret_cast<const float4 *>(rope_row)[lane];  // c0 s0 c1 s1
+    const float2 ra = make_float2(a.x * cs.x - b.x * cs.y, a.y * cs.z - b.y * cs.w);
+    const float2 rb = make_float2(b.x * cs.x + a.x * cs.y, b.y * cs.z + a.y * cs.w);
+    a = ra; b = rb;
+}
+
+template <int G, bool FUSED>
+__global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(const AttnParams p) {
+    NNC_TRACE_SCOPE(30);
+    __shared__ __align__(16) float qs[G][kHeadDim];              // processed queries, pre-scaled for exp2
+    __shared__ float comb[kWarps][G][kPartStride];               // per-warp (o~, m, l)
     __shared__ bool is_last;
 
-    pdl_wait();
     const int split = blockIdx.x, j = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slot = tid >> 4;   // 8 position slots
-    const int dl = tid & 15;     // 16-byte slice of the head dimension
-    const int n_ctx = (d_len ? *d_len : 0) + len_add;
-    const int nq = nkv * G;
-    int chunk = (n_ctx + n_splits - 1) / n_splits;
+    const int g8 = lane >> 2, t4 = lane & 3;   // fragment coordinates: row / column group, and position inside it
+    const int nq = p.nkv * G;
+    const size_t head_off = ((size_t)b * p.nkv + j) * (size_t)p.max_seq * kHeadDim;
+    bf16 *kbase = p.kcache + head_off;
+    bf16 *vbase = p.vcache + head_off;
+
+    pdl_launch_dependents();
+    // ---- before the dependency: ask for this CTA's K/V range in L2 (rows of earlier positions are stable) ----
+    {
+        const int n_guess = (p.d_len ? *p.d_len : 0) + p.len_add;   // only a hint here; read again after the wait
+        int chunk = (n_guess + p.n_splits - 1) / p.n_splits;
+        chunk = (chunk + 15) & ~15;
+        if (chunk < 16) chunk = 16;
+        const int c0 = split * chunk, c1 = min(c0 + chunk, min(n_guess, p.max_seq));
+        if (tid < 2 && c1 > c0) {
+            const bf16 *src = (tid ? vbase : kbase) + (size_t)c0 * kHeadDim;
+            const uint32_t bytes = (uint32_t)(c1 - c0) * kHeadDim * 2u;
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+        }
+    }
+    pdl_wait();
+    NNC_TRACE_MARK();
+
+    const int n_ctx = (p.d_len ? *p.d_len : 0) + p.len_add;
+    int chunk = (n_ctx + p.n_splits - 1) / p.n_splits;
     chunk = (chunk + 15) & ~15;
     if (chunk < 16) chunk = 16;
     const int c0 = split * chunk;
@@ -49,160 +124,226 @@ attn_decode_kernel(const float *__restrict__ q, int q_row_stride, const bf16 *__
     const int n_active = (n_ctx + chunk - 1) / chunk;
     if (c0 >= n_ctx) return;  // whole CTA; takes no ticket (n_active counts only non-empty ranges)
 
-    // query slice in registers, pre-scaled so that exp2 can be used: s' = s * log2(e) / sqrt(d)
-    const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
-    float qr[G][8];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-        const float *qp = q + (size_t)b * q_row_stride + (size_t)(j * G + g) * kHeadDim + dl * 8;
-        const float4 a = reinterpret_cast<const float4 *>(qp)[0], c = reinterpret_cast<const float4 *>(qp)[1];
-        qr[g][0] = a.x * qscale; qr[g][1] = a.y * qscale; qr[g][2] = a.z * qscale; qr[g][3] = a.w * qscale;
-        qr[g][4] = c.x * qscale; qr[g][5] = c.y * qscale; qr[g][6] = c.z * qscale; qr[g][7] = c.w * qscale;
+    // ---- queries (and, fused, the new token's K/V row) ----
+    const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);   // scores in log2 units
+    const float *qrow = p.q + (size_t)b * p.q_row_stride;
+    for (int g = warp; g < G; g += kWarps) {
+        const float *src = qrow + (size_t)(j * G + g) * kHeadDim;
+        float2 a = reinterpret_cast<const float2 *>(src)[lane];
+        float2 c = reinterpret_cast<const float2 *>(src + 64)[lane];
+        if (FUSED) norm_rope(a, c, p.g_q, p.rope + (size_t)(n_ctx - 1) * kHeadDim, p.eps, lane);
+        reinterpret_cast<float2 *>(&qs[g][0])[lane] = make_float2(a.x * qscale, a.y * qscale);
+        reinterpret_cast<float2 *>(&qs[g][64])[lane] = make_float2(c.x * qscale, c.y * qscale);
     }
-    if (tid < G) { s_m[tid] = -INFINITY; s_l[tid] = 0.f; }
-
-    const size_t head_off = ((size_t)b * nkv + j) * (size_t)max_seq * kHeadDim;
-    const bf16 *kbase = kcache + head_off + dl * 8;
-    const bf16 *vbase = vcache + head_off + dl * 8;
-
-    float acc[G][8];
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
-
-    for (int t0 = c0; t0 < c1; t0 += kTile) {
-        // ---- scores of this tile ----
-#pragma unroll 4
-        for (int it = 0; it < kTile / 8; ++it) {
-            const int p = t0 + it * 8 + slot;
-            float s[G];
-            if (p < c1) {
-                float kf[8];
-                unpack8(ldg_stream(kbase + (size_t)p * kHeadDim), kf);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float d = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) d = fmaf(qr[g][i], kf[i], d);
-                    s[g] = d;
-                }
-            } else {
-#pragma unroll
-                for (int g = 0; g < G; ++g) s[g] = 0.f;
-            }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) s[g] += __shfl_xor_sync(0xffffffffu, s[g], o);
-            }
-            if (dl == 0) {
-#pragma unroll
-                for (int g = 0; g < G; ++g) sc[g][it * 8 + slot] = p < c1 ? s[g] : -INFINITY;
-            }
+    if (FUSED && split == n_active - 1) {
+        // this CTA's range ends with the new position: normalise + rotate its key, round both rows to bf16, append
+        const int pos = n_ctx - 1;
+        if (warp == (G % kWarps)) {
+            const float *src = qrow + (size_t)(nq + j) * kHeadDim;
+            float2 a = reinterpret_cast<const float2 *>(src)[lane];
+            float2 c = reinterpret_cast<const float2 *>(src + 64)[lane];
+            norm_rope(a, c, p.g_k, p.rope + (size_t)pos * kHeadDim, p.eps, lane);
+            bf16 *dst = kbase + (size_t)pos * kHeadDim;
+            reinterpret_cast<uint32_t *>(dst)[lane] = pack_bf16x2(a.x, a.y);
+            reinterpret_cast<uint32_t *>(dst + 64)[lane] = pack_bf16x2(c.x, c.y);
         }
-        __syncthreads();
-        // ---- online softmax bookkeeping: warp w handles heads w, w+4 ----
-        for (int g = warp; g < G; g += 4) {
-            float mx = -INFINITY;
-#pragma unroll
-            for (int i = lane; i < kTile; i += 32) mx = fmaxf(mx, sc[g][i]);
-            mx = warp_max(mx);
-            const float m_old = s_m[g];
-            const float m_new = fmaxf(m_old, mx);  // finite: the tile holds at least one valid position
-            float sum = 0.f;
-#pragma unroll
-            for (int i = lane; i < kTile; i += 32) {
-                const float pr = exp2f(sc[g][i] - m_new);
-                sc[g][i] = pr;
-                sum += pr;
-            }
-            sum = warp_sum(sum);
-            if (lane == 0) {
-                const float alpha = exp2f(m_old - m_new);  // 0 on the first tile
-                s_alpha[g] = alpha;
-                s_l[g] = s_l[g] * alpha + sum;
-                s_m[g] = m_new;
-            }
+        if (warp == ((G + 1) % kWarps)) {
+            const float *src = qrow + (size_t)(nq + p.nkv + j) * kHeadDim;
+            const float4 v = reinterpret_cast<const float4 *>(src)[lane];
+            bf16 *dst = vbase + (size_t)pos * kHeadDim;
+            reinterpret_cast<uint2 *>(dst)[lane] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
         }
-        __syncthreads();
-        // ---- o~ = o~ * alpha + P V ----
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float al = s_alpha[g];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[g][i] *= al;
-        }
-#pragma unroll 4
-        for (int it = 0; it < kTile / 8; ++it) {
-            const int p = t0 + it * 8 + slot;
-            if (p < c1) {
-                float vf[8];
-                unpack8(ldg_stream(vbase + (size_t)p * kHeadDim), vf);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const float pr = sc[g][it * 8 + slot];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(pr, vf[i], acc[g][i]);
-                }
-            }
-        }
-        __syncthreads();
-    }
-
-    // ---- fold the 8 position slots: lanes 16 apart, then the 4 warps ----
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] += __shfl_xor_sync(0xffffffffu, acc[g][i], 16);
-    if (lane < 16) {
-#pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) red[warp][g][dl * 8 + i] = acc[g][i];
+        __threadfence_block();
     }
     __syncthreads();
-    pdl_launch_dependents();
 
-    float *my_part = part + (((size_t)b * nq + (size_t)j * G) * n_splits + split) * kPartStride;
+    // ---- Q fragments: row g8 (a query head, zero beyond G), contraction step s = 2c + e covers the head-dimension
+    //      elements 8 (4c + t4) + 4e + {0,1} (first half of the step) and + {2,3} (second half) ----
+    uint32_t qh[8][2], ql[8][2];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f), hi4 = lo4;
+        if (g8 < G) {
+            lo4 = *reinterpret_cast<const float4 *>(&qs[g8 < G ? g8 : 0][8 * (4 * c + t4)]);
+            hi4 = *reinterpret_cast<const float4 *>(&qs[g8 < G ? g8 : 0][8 * (4 * c + t4) + 4]);
+        }
+        split2(lo4.x, lo4.y, qh[2 * c][0], ql[2 * c][0]);
+        split2(lo4.z, lo4.w, qh[2 * c][1], ql[2 * c][1]);
+        split2(hi4.x, hi4.y, qh[2 * c + 1][0], ql[2 * c + 1][0]);
+        split2(hi4.z, hi4.w, qh[2 * c + 1][1], ql[2 * c + 1][1]);
+    }
+
+    float o[16][4];   // output tile j2: columns n = 2 t4, 2 t4 + 1 of row g8 in [0], [1]; [2], [3] belong to padding rows
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run = -INFINITY, l_run = 0.f;   // per row g8 (identical across the 4 lanes of a row); l is a per-lane partial
+
+    const int n_blocks = (c1 - c0 + 15) >> 4;
+    for (int blk = warp; blk < n_blocks; blk += kWarps) {
+        const int p0 = c0 + blk * 16;
+        // ---- loads: K rows p0 + 8h + g8 (h = 0, 1), V rows p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9} ----
+        uint4 kf[2][4], vf[4][2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int pos = min(p0 + 8 * h + g8, c1 - 1);   // rows past the range are clamped and masked below
+            const bf16 *kr = kbase + (size_t)pos * kHeadDim + 8 * t4;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) kf[h][c] = ldg_cg(kr + 32 * c);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int pos = min(p0 + 2 * t4 + (r & 1) + 8 * (r >> 1), c1 - 1);
+            const bf16 *vr = vbase + (size_t)pos * kHeadDim + 8 * g8;
+            vf[r][0] = ldg_cg(vr);
+            vf[r][1] = ldg_cg(vr + 64);
+        }
+        // ---- scores: S[h] = Q K^T for the 8 positions of half h ----
+        float s[2][4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            s[h][0] = s[h][1] = s[h][2] = s[h][3] = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t r0 = kf[h][c].x, r1 = kf[h][c].y, r2 = kf[h][c].z, r3 = kf[h][c].w;
+                mma_bf16(s[h], qh[2 * c][0], qh[2 * c][1], r0, r1);
+                mma_bf16(s[h], ql[2 * c][0], ql[2 * c][1], r0, r1);
+                mma_bf16(s[h], qh[2 * c + 1][0], qh[2 * c + 1][1], r2, r3);
+                mma_bf16(s[h], ql[2 * c + 1][0], ql[2 * c + 1][1], r2, r3);
+            }
+        }
+        // this lane holds row g8, positions p0 + 8h + 2 t4 + {0, 1}
+        float mx = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (p0 + 8 * h + 2 * t4 + e >= c1) s[h][e] = -INFINITY;
+                mx = fmaxf(mx, s[h][e]);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);           // finite: the block holds at least one valid position
+        const float alpha = exp2f(m_run - m_new);       // 0 on the first block
+        float pr[2][2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) pr[h][e] = exp2f(s[h][e] - m_new);
+        l_run = l_run * alpha + (pr[0][0] + pr[0][1] + pr[1][0] + pr[1][1]);
+        m_run = m_new;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
+        // ---- P fragments (contraction index = position inside the block), as value + residual ----
+        uint32_t ph0, pl0, ph1, pl1;
+        split2(pr[0][0], pr[0][1], ph0, pl0);   // positions 2 t4, 2 t4 + 1
+        split2(pr[1][0], pr[1][1], ph1, pl1);   // positions 2 t4 + 8, 2 t4 + 9
+        // ---- O += P V: output tile i covers head-dimension element (i < 8 ? 8 n + i : 64 + 8 n + i - 8), n = column ----
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int q2 = i >> 3, e = i & 7;
+            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+            const uint32_t ra = (&vf[0][q2].x)[e >> 1], rb = (&vf[1][q2].x)[e >> 1];
+            const uint32_t rc = (&vf[2][q2].x)[e >> 1], rd = (&vf[3][q2].x)[e >> 1];
+            const uint32_t b0 = prmt(ra, rb, sel), b1 = prmt(rc, rd, sel);
+            mma_bf16(o[i], ph0, ph1, b0, b1);
+            mma_bf16(o[i], pl0, pl1, b0, b1);
+        }
+    }
+
+    NNC_TRACE_MARK2();
+    // ---- merge the warps: (o~, m, l) per query head into shared memory, then one partial per CTA ----
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (g8 < G) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int d0 = (i < 8) ? 8 * (2 * t4) + i : 64 + 8 * (2 * t4) + (i - 8);
+            comb[warp][g8][d0] = o[i][0];
+            comb[warp][g8][d0 + 8] = o[i][1];
+        }
+        if (t4 == 0) { comb[warp][g8][kHeadDim] = m_run; comb[warp][g8][kHeadDim + 1] = l_run; }
+    }
+    __syncthreads();
+
+    float *my_part = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits + split) * kPartStride;
     // partial for head g lives at my_part + g * n_splits * kPartStride
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        float *pp = my_part + (size_t)g * n_splits * kPartStride;
-        pp[tid] = red[0][g][tid] + red[1][g][tid] + red[2][g][tid] + red[3][g][tid];
-        if (tid == 0) { pp[kHeadDim] = s_m[g]; pp[kHeadDim + 1] = s_l[g]; }
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, comb[w][g][kHeadDim]);
+        float L = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float sc = exp2f(comb[w][g][kHeadDim] - M);   // 0 for a warp that had no block
+            L = fmaf(sc, comb[w][g][kHeadDim + 1], L);
+            acc = fmaf(sc, comb[w][g][tid], acc);
+        }
+        float *pp = my_part + (size_t)g * p.n_splits * kPartStride;
+        pp[tid] = acc;
+        if (tid == 0) { pp[kHeadDim] = M; pp[kHeadDim + 1] = L; }
     }
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned t = atomicAdd(&tickets[b * nkv + j], 1u);
-        is_last = (t == (unsigned)n_active - 1);
+        const unsigned tk = atomicAdd(&p.tickets[b * p.nkv + j], 1u);
+        is_last = (tk == (unsigned)n_active - 1);
     }
     __syncthreads();
+    NNC_TRACE_MARK3();
     if (!is_last) return;
     __threadfence();
-    // ---- combine (last CTA of this sequence / KV head): o = sum_c 2^(m_c - M) o~_c / sum_c 2^(m_c - M) l_c ----
+    // ---- combine (last CTA of this sequence / KV head): o = sum_c 2^(m_c - M) o~_c / sum_c 2^(m_c - M) l_c.
+    //      Weights first (one warp per head, splits across lanes), then every thread folds its output element
+    //      over the splits with all loads of a batch of splits in flight at once. ----
+    float (*wgt)[kAttnMaxSplits] = reinterpret_cast<float (*)[kAttnMaxSplits]>(&comb[0][0][0]);   // [G][kAttnMaxSplits], reuses comb
+    __shared__ float inv_l[G];
+    const float *pbase = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits) * kPartStride;
+    for (int g = warp; g < G; g += kWarps) {
+        const float *pp = pbase + (size_t)g * p.n_splits * kPartStride;
+        float mv[2], lv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int c = lane + 32 * u;
+            mv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim) : -INFINITY;
+            lv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim + 1) : 0.f;
+        }
+        const float M = warp_max(fmaxf(mv[0], mv[1]));
+        const float w0 = exp2f(mv[0] - M), w1 = exp2f(mv[1] - M);
+        wgt[g][lane] = w0;
+        wgt[g][lane + 32] = w1;
+        // fixed summation order over the splits: lane partials, then the shuffle tree
+        const float L = warp_sum(fmaf(w0, lv[0], w1 * lv[1]));
+        if (lane == 0) inv_l[g] = 1.f / L;
+    }
+    __syncthreads();
+    float acc[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) acc[g] = 0.f;
+    for (int cb = 0; cb < n_active; cb += 8) {
+        float v[G][8];
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[g][u] = (cb + u < n_active) ? __ldcg(pbase + ((size_t)g * p.n_splits + cb + u) * kPartStride + tid) : 0.f;
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc[g] = fmaf(cb + u < n_active ? wgt[g][cb + u] : 0.f, v[g][u], acc[g]);
+    }
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        const volatile float *pp = part + (((size_t)b * nq + (size_t)j * G + g) * n_splits) * kPartStride;
-        float M = -INFINITY;
-        for (int c = 0; c < n_active; ++c) M = fmaxf(M, pp[(size_t)c * kPartStride + kHeadDim]);
-        float L = 0.f, o = 0.f;
-        for (int c = 0; c < n_active; ++c) {
-            const float w = exp2f(pp[(size_t)c * kPartStride + kHeadDim] - M);
-            L = fmaf(w, pp[(size_t)c * kPartStride + kHeadDim + 1], L);
-            o = fmaf(w, pp[(size_t)c * kPartStride + tid], o);
-        }
-        const float r = o / L;
-        const size_t oi = (size_t)b * out_row_stride + (size_t)(j * G + g) * kHeadDim + tid;
-        if (out_f32) out_f32[oi] = r;
-        if (out_bf16) {
+        const float r = acc[g] * inv_l[g];
+        const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + tid;
+        if (p.out_f32) p.out_f32[oi] = r;
+        if (p.out_bf16) {
             const bf16 hi = __float2bfloat16_rn(r);
-            out_bf16[oi] = hi;
-            if (out_bf16_lo) out_bf16_lo[oi] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            p.out_bf16[oi] = hi;
+            if (p.out_bf16_lo) p.out_bf16_lo[oi] = __float2bfloat16_rn(r - __bfloat162float(hi));
         }
     }
-    if (tid == 0) tickets[b * nkv + j] = 0u;
+    if (tid == 0) p.tickets[b * p.nkv + j] = 0u;
 }
 
 }  // namespace
@@ -221,17 +362,23 @@ size_t attn_decode_scratch_floats(int batch, int nq, int n_splits) {
     return (size_t)batch * nq * n_splits * kPartStride;
 }
 
-cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, const bf16 *kcache,
-                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride,
-                               float *part,
+cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, bf16 *kcache, bf16 *vcache,
+                               float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride, float *part,
                                uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
-                               int max_seq, int n_splits) {
+                               int max_seq, int n_splits, const AttnFused *fused) {
     const int G = nq / nkv;
-    dim3 grid(n_splits, nkv, batch), block(128);
-#define NNC_ATTN_CASE(GG)                                                                                       \
-    case GG:                                                                                                    \
-        return launch(lc, attn_decode_kernel<GG>, grid, block, q, q_row_stride, kcache, vcache, out_f32,       \
-                      out_bf16, out_bf16_lo, out_row_stride, part, tickets, d_len, len_add, nkv, max_seq, n_splits);
+    AttnParams p;
+    p.q = q; p.q_row_stride = q_row_stride; p.kcache = kcache; p.vcache = vcache;
+    p.out_f32 = out_f32; p.out_bf16 = out_bf16; p.out_bf16_lo = out_bf16_lo; p.out_row_stride = out_row_stride;
+    p.part = part; p.tickets = tickets; p.d_len = d_len; p.len_add = len_add;
+    p.nkv = nkv; p.max_seq = max_seq; p.n_splits = n_splits;
+    p.g_q = fused ? fused->g_q : nullptr; p.g_k = fused ? fused->g_k : nullptr;
+    p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;
+    dim3 grid(n_splits, nkv, batch), block(kWarps * 32);
+#define NNC_ATTN_CASE(GG)                                                                  \
+    case GG:                                                                               \
+        return fused ? launch(lc, attn_decode_kernel<GG, true>, grid, block, p)           \
+                     : launch(lc, attn_decode_kernel<GG, false>, grid, block, p);
     switch (G) {
         NNC_ATTN_CASE(1)
         NNC_ATTN_CASE(2)

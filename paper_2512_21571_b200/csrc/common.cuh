@@ -49,4 +49,46 @@ __device__ __forceinline__ float warp_max(float v) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- per-CTA timeline records (tracing builds only: -DNNC_TRACE) -----------------------------------------
+// Every CTA appends {kernel id, block, SM, start, end} (globaltimer ns) to a device buffer when it exits;
+// nnc_trace_dump() copies the buffer to the host.  Compiled out of the normal library.  Each translation unit
+// holds its own copy of the two pointers (no relocatable device code) and registers a binder for them.
+#ifdef NNC_TRACE
+struct TraceRec { unsigned kid, block, smid, mark; unsigned long long t0, t1; unsigned mark2, mark3, pad0, pad1; };
+constexpr unsigned kTraceMax = 1u << 20;
+static __device__ TraceRec *g_trace_buf;
+static __device__ unsigned *g_trace_cnt;
+void trace_register(void (*bind)(TraceRec *, unsigned *));
+static void trace_bind_this_tu(TraceRec *buf, unsigned *cnt) {
+    cudaMemcpyToSymbol(g_trace_buf, &buf, sizeof(buf));
+    cudaMemcpyToSymbol(g_trace_cnt, &cnt, sizeof(cnt));
+}
+namespace { struct TraceRegistrar { TraceRegistrar() { trace_register(&trace_bind_this_tu); } } g_trace_registrar; }
+struct TraceScope {
+    unsigned kid, mark, mark2, mark3; unsigned long long t0;
+    __device__ __forceinline__ unsigned since() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned)(t - t0); }
+    __device__ __forceinline__ void set_mark() { mark = since(); }
+    __device__ __forceinline__ void set_mark2() { mark2 = since(); }
+    __device__ __forceinline__ void set_mark3() { mark3 = since(); }
+    __device__ __forceinline__ TraceScope(unsigned k) : kid(k), mark(0), mark2(0), mark3(0) { asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0)); }
+    __device__ __forceinline__ ~TraceScope() {
+        if (threadIdx.x == 0 && g_trace_buf) {
+            unsigned long long t1; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+            unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+            const unsigned i = atomicAdd(g_trace_cnt, 1u);
+            if (i < kTraceMax) g_trace_buf[i] = TraceRec{kid, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), sm, mark, t0, t1, mark2, mark3, 0, 0};
+        }
+    }
+};
+#define NNC_TRACE_SCOPE(kid) TraceScope nnc_trace_scope__(kid)
+#define NNC_TRACE_MARK() nnc_trace_scope__.set_mark()
+#define NNC_TRACE_MARK2() nnc_trace_scope__.set_mark2()
+#define NNC_TRACE_MARK3() nnc_trace_scope__.set_mark3()
+#else
+#define NNC_TRACE_SCOPE(kid)
+#define NNC_TRACE_MARK()
+#define NNC_TRACE_MARK2()
+#define NNC_TRACE_MARK3()
+#endif
+
 }  // namespace nnc

@@ -38,6 +38,7 @@ template <int ROWS, int MODE, bool NORM>
 __global__ void __launch_bounds__(kGemvThreads)
 gemv_kernel(const uint4 *__restrict__ W, const float *__restrict__ x, float *__restrict__ y, int n_out, int n_in,
             const bf16 *__restrict__ gain, float eps, ArgmaxScratch am) {
+    NNC_TRACE_SCOPE(20 + MODE);
     extern __shared__ float4 xs[];  // two planes of n_in/8 float4: plane h holds elements 8c+4h .. 8c+4h+3 of chunk c
     __shared__ float red[kGemvWarps];
     __shared__ int red_i[kGemvWarps];
@@ -243,6 +244,7 @@ cudaError_t launch_rows(const LaunchCtx &lc, const bf16 *W, const float *x, floa
 
 cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
                         const bf16 *gain, float eps, int mode, const ArgmaxScratch *am) {
+    if (gemv_stream_supported(n_out, n_in, mode)) return launch_gemv_stream(lc, W, x, y, n_out, n_in, gain, eps, mode, am);
     if (n_in % 8 != 0 || n_in <= 0 || n_out <= 0 || (size_t)n_in * 4 > 200 * 1024) return cudaErrorInvalidValue;
     ArgmaxScratch a = am ? *am : ArgmaxScratch{nullptr, nullptr, nullptr, nullptr};
     const bool norm = gain != nullptr;

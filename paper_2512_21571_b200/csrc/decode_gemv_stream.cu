@@ -1,0 +1,459 @@
+// Batch-1 decode GEMV, streaming form: y = W x for a bf16 matrix W[n_out][K] read exactly once from HBM.
+//
+// HBM-bound (1 FLOP per weight byte), so the kernel is built around bytes in flight, not arithmetic:
+//   - one persistent CTA per SM: a producer warp and 8 consumer warps around a shared-memory ring.  The producer
+//     keeps the ring full with cp.async.bulk copies (the 1-D form of TMA) of 8-32 KB each -- whole consecutive
+//     rows, which are contiguous in the row-major matrix -- so ~100 KB per SM are outstanding without holding
+//     registers, and each copy is large enough that the copy engine's request rate is not the limit;
+//   - the matrix is cut into stages of `rps` rows and every CTA takes an equal contiguous run of stages
+//     (~14 or more per SM whatever the shape: no wave quantisation);
+//   - inside a stage `ksplit` warps share a row, each taking a contiguous K slice whose activations it holds in
+//     registers (optionally RMS-normalised on the way in), so shared memory carries weights only;
+//   - per-row partial sums meet in a small double-buffered shared array and are folded in fixed order every
+//     ~64 rows (deterministic: no float atomics), where the epilogue runs: store, residual add, SwiGLU on
+//     interleaved gate/up rows, or logits + arg-max candidates (the last CTA folds those; nobody waits);
+//   - launched with programmatic stream serialization: dependents are released at once and the producer never
+//     waits on the previous kernel (weights depend on nothing), so a CTA starts streaming the moment its SM is
+//     free.  The ring takes more than half of an SM's shared memory on purpose: two of these CTAs can never share
+//     an SM, so each kernel's 148 CTAs land one per SM (with smaller rings the block scheduler was seen to stack
+//     two CTAs of one kernel on some SMs and leave others idle whenever the previous kernel still held space).
+// Every mbarrier wait is bounded; on expiry the CTA raises the status word and drains.
+#include <stdio.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+#include "nnc_internal.h"
+
+namespace nnc {
+
+namespace {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;   // + the producer warp
+constexpr int kMaxStages = 12;
+constexpr int kRingBytes = 192 * 1024;          // more than half an SM: exactly one of these CTAs fits per SM
+constexpr int kBlockRows = 64;                    // rows between two folds of the partial sums
+constexpr uint32_t kSpinLimit = 1u << 22;         // try_wait attempts before a wait gives up (each may block ~us)
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 w;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "r"(addr));
+    return w;
+}
+
+// dot product of J 16-byte weight chunks with the matching activations: 2 J independent FMA chains
+template <int J>
+__device__ __forceinline__ float dot_slice(const uint4 (&w)[J], const float (&xr)[J][8]) {
+    float a[J][2];
+#pragma unroll
+    for (int i = 0; i < J; ++i) {
+        a[i][0] = bf16_lo(w[i].x) * xr[i][0];
+        a[i][1] = bf16_hi(w[i].x) * xr[i][1];
+        a[i][0] = fmaf(bf16_lo(w[i].y), xr[i][2], a[i][0]);
+        a[i][1] = fmaf(bf16_hi(w[i].y), xr[i][3], a[i][1]);
+        a[i][0] = fmaf(bf16_lo(w[i].z), xr[i][4], a[i][0]);
+        a[i][1] = fmaf(bf16_hi(w[i].z), xr[i][5], a[i][1]);
+        a[i][0] = fmaf(bf16_lo(w[i].w), xr[i][6], a[i][0]);
+        a[i][1] = fmaf(bf16_hi(w[i].w), xr[i][7], a[i][1]);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < J; ++i) s += a[i][0] + a[i][1];
+    return s;
+}
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
+
+struct StreamParams {
+    const uint8_t *W;
+    const float *x;
+    float *y;
+    const bf16 *gain;
+    float eps;
+    int n_out, K;
+    int ksplit;    // consumer warps per row (1, 2, 4, 8)
+    int kw;        // columns of a warp's slice = K / ksplit (multiple of 8)
+    int rps;       // rows per stage (a multiple of 8 / ksplit)
+    int stages;    // ring depth
+    int n_stages;  // stages in the whole matrix = ceil(n_out / rps)
+    int pb;        // stages per fold block = kBlockRows / rps (at least 1)
+    int *status;   // raised if a bounded wait runs out
+    ArgmaxScratch am;
+};
+
+// J = 16-byte chunks per lane per row slice (kw <= J * 256).
+template <int J, int MODE, bool NORM>
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
+    NNC_TRACE_SCOPE(10 + MODE + 100 * (p.K / 1024));
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ __align__(8) uint64_t full[kMaxStages], empty[kMaxStages];
+    __shared__ float part[2][kBlockRows][kConsumerWarps];
+    __shared__ float red[kConsumerWarps];
+    __shared__ int red_i[kConsumerWarps];
+    __shared__ bool is_last;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages;
+    const uint32_t row_bytes = (uint32_t)p.K * 2u;
+    const uint32_t stage_bytes = (uint32_t)p.rps * row_bytes;
+
+    const int per = p.n_stages / gridDim.x, rem = p.n_stages % gridDim.x;
+    const int st0 = blockIdx.x * per + min((int)blockIdx.x, rem);
+    const int n_st = per + ((int)blockIdx.x < rem ? 1 : 0);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&full[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&empty[s])), "r"(kConsumerWarps));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer: streams this CTA's stages; never waits on the previous kernel ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int s = 0; s < n_st; ++s) {
+                if (!mbar_wait_bounded(smem_u32(&empty[stage]), phase ^ 1u)) {
+                    if (p.status) atomicExch(p.status, 17);
+                    break;
+                }
+                const int row0 = (st0 + s) * p.rps;
+                const int rows = min(p.rps, p.n_out - row0);
+                bulk_load(smem_u32(ring) + (uint32_t)stage * stage_bytes, p.W + (size_t)row0 * row_bytes,
+                          (uint32_t)rows * row_bytes, smem_u32(&full[stage]));
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    const int ksplit = p.ksplit, gpi = kConsumerWarps / ksplit;
+    const int ks = warp % ksplit, gi = warp / ksplit;
+    const int rw = p.rps / gpi;   // rows this warp owns in each stage: gi, gi + gpi, ...
+    // gains are weights: fetch them before waiting on the kernel that produces x
+    uint4 gr[NORM ? J : 1];
+    if (NORM) {
+#pragma unroll
+        for (int i = 0; i < J; ++i) {
+            const int c = lane + 32 * i;
+            gr[i] = (c * 8 < p.kw) ? *reinterpret_cast<const uint4 *>(p.gain + (size_t)ks * p.kw + (size_t)c * 8) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    pdl_wait();
+    NNC_TRACE_MARK();
+
+    // this warp's activation slice, in registers
+    float xr[J][8];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < J; ++i) {
+        const int c = lane + 32 * i;
+        if (c * 8 < p.kw) {
+            const float4 *xp = reinterpret_cast<const float4 *>(p.x + (size_t)ks * p.kw + (size_t)c * 8);
+            const float4 a = xp[0], b = xp[1];
+            xr[i][0] = a.x; xr[i][1] = a.y; xr[i][2] = a.z; xr[i][3] = a.w;
+            xr[i][4] = b.x; xr[i][5] = b.y; xr[i][6] = b.z; xr[i][7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) xr[i][e] = 0.f;
+        }
+        if (NORM) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
+        }
+    }
+    if (NORM) {
+        ss = warp_sum(ss);
+        if (lane == 0) red[warp] = ss;
+        consumer_sync();
+        float tot = 0.f;
+        for (int k = 0; k < ksplit; ++k) tot += red[k];   // warps 0 .. ksplit-1 hold the ksplit distinct slices
+        const float inv = rsqrtf(tot / (float)p.K + p.eps);
+#pragma unroll
+        for (int i = 0; i < J; ++i) {
+            const int c = lane + 32 * i;
+            {
+                const uint4 g = gr[i];
+                xr[i][0] *= inv * bf16_lo(g.x); xr[i][1] *= inv * bf16_hi(g.x);
+                xr[i][2] *= inv * bf16_lo(g.y); xr[i][3] *= inv * bf16_hi(g.y);
+                xr[i][4] *= inv * bf16_lo(g.z); xr[i][5] *= inv * bf16_hi(g.z);
+                xr[i][6] *= inv * bf16_lo(g.w); xr[i][7] *= inv * bf16_hi(g.w);
+            }
+        }
+        consumer_sync();   // red is reused by the arg-max fold
+    }
+
+    float best_v = -INFINITY;
+    int best_i = 0x7fffffff;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    const uint32_t slice_off = (uint32_t)ks * (uint32_t)p.kw * 2u;
+
+    for (int b0 = 0, blk = 0; b0 < n_st; b0 += p.pb, ++blk) {
+        const int nb = min(p.pb, n_st - b0);
+        const int buf = blk & 1;
+        const int block_row0 = (st0 + b0) * p.rps;
+        const int rows_here = min(nb * p.rps, p.n_out - block_row0);
+        float y_old = 0.f;   // residual mode: fetched now, used at the fold (hides the global-load latency)
+        if (MODE == kGemvResidual && (int)threadIdx.x < rows_here) y_old = p.y[block_row0 + threadIdx.x];
+        for (int j = 0; j < nb; ++j) {
+            if (ok && !mbar_wait_bounded(smem_u32(&full[stage]), phase)) {
+                ok = false;
+                if (lane == 0 && p.status) atomicExch(p.status, 16);
+            }
+            const uint32_t sbase = smem_u32(ring) + (uint32_t)stage * stage_bytes + slice_off;
+            // rows of this stage owned by the warp, two at a time (independent load / FMA streams, one joint reduction)
+            for (int m = 0; m < rw && ok; m += 2) {
+                const int r_in_stage = gi + gpi * m;
+                const int r_in_block = j * p.rps + r_in_stage;
+                if (block_row0 + r_in_block >= p.n_out) break;   // ragged last stage (warp-uniform)
+                const bool two = (m + 1 < rw) && (block_row0 + r_in_block + gpi < p.n_out);
+                const uint32_t rbase0 = sbase + (uint32_t)r_in_stage * row_bytes;
+                const uint32_t rbase1 = two ? rbase0 + (uint32_t)gpi * row_bytes : rbase0;
+                uint4 w0[J], w1[J];
+#pragma unroll
+                for (int i = 0; i < J; ++i) {
+                    const int c = lane + 32 * i;
+                    w0[i] = make_uint4(0, 0, 0, 0);
+                    w1[i] = make_uint4(0, 0, 0, 0);
+                    if (c * 8 < p.kw) {
+                        w0[i] = lds128(rbase0 + (uint32_t)c * 16u);
+                        w1[i] = lds128(rbase1 + (uint32_t)c * 16u);
+                    }
+                }
+                float s0 = dot_slice<J>(w0, xr), s1 = dot_slice<J>(w1, xr);
+                // joint reduction: lanes 0-15 end up with row 0, lanes 16-31 with row 1
+                const bool upper = (lane & 16) != 0;
+                float keep = upper ? s1 : s0;
+                keep += __shfl_xor_sync(0xffffffffu, upper ? s0 : s1, 16);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) keep += __shfl_xor_sync(0xffffffffu, keep, o);
+                if (lane == 0) part[buf][r_in_block][ks] = keep;
+                if (lane == 16 && two) part[buf][r_in_block + gpi][ks] = keep;
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[stage])) : "memory");
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        consumer_sync();
+        // ---- fold the ksplit partial sums of each row in fixed order; epilogue ----
+        const int t = threadIdx.x;
+        if (MODE == kGemvSwiglu) {
+            if (2 * t + 1 < rows_here) {
+                float g = 0.f, u = 0.f;
+                for (int k = 0; k < ksplit; ++k) { g += part[buf][2 * t][k]; u += part[buf][2 * t + 1][k]; }
+                p.y[(block_row0 >> 1) + t] = g / (1.f + __expf(-g)) * u;
+            }
+        } else if (t < rows_here) {
+            float v = 0.f;
+            for (int k = 0; k < ksplit; ++k) v += part[buf][t][k];
+            const int row = block_row0 + t;
+            if (MODE == kGemvResidual) v += y_old;
+            p.y[row] = v;
+            if (MODE == kGemvLogits && better(v, row, best_v, best_i)) { best_v = v; best_i = row; }
+        }
+    }
+
+    if (MODE == kGemvLogits && p.am.out != nullptr) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best_v, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+            if (better(ov, oi, best_v, best_i)) { best_v = ov; best_i = oi; }
+        }
+        if (lane == 0) { red[warp] = best_v; red_i[warp] = best_i; }
+        consumer_sync();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < kConsumerWarps; ++w)
+                if (better(red[w], red_i[w], best_v, best_i)) { best_v = red[w]; best_i = red_i[w]; }
+            p.am.part_val[blockIdx.x] = best_v;
+            p.am.part_idx[blockIdx.x] = best_i;
+            __threadfence();
+            const unsigned tk = atomicAdd(p.am.ticket, 1u);
+            is_last = (tk == gridDim.x - 1);
+        }
+        consumer_sync();
+        if (is_last) {  // the CTA that arrives last folds every CTA's candidate; nobody waits
+            __threadfence();
+            float bv = -INFINITY;
+            int bi = 0x7fffffff;
+            for (int b = threadIdx.x; b < (int)gridDim.x; b += kConsumerThreads) {
+                const float v = ((volatile float *)p.am.part_val)[b];
+                const int i = ((volatile int *)p.am.part_idx)[b];
+                if (better(v, i, bv, bi)) { bv = v; bi = i; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+            }
+            consumer_sync();
+            if (lane == 0) { red[warp] = bv; red_i[warp] = bi; }
+            consumer_sync();
+            if (threadIdx.x == 0) {
+                for (int w = 1; w < kConsumerWarps; ++w)
+                    if (better(red[w], red_i[w], bv, bi)) { bv = red[w]; bi = red_i[w]; }
+                *p.am.out = bi == 0x7fffffff ? 0 : bi;
+                *p.am.ticket = 0u;
+            }
+        }
+    }
+    if (!ok) {
+        // a copy never signalled: give whatever is still in flight time to land before shared memory is released
+        for (int s = 0; s < 64; ++s) __nanosleep(1000);
+    }
+}
+
+template <int J, int MODE, bool NORM>
+cudaError_t launch_j(const LaunchCtx &lc, const StreamParams &p, int grid, size_t smem) {
+    auto kern = gemv_stream_kernel<J, MODE, NORM>;
+    static bool attr_done = false;  // per instantiation
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    if (lc.launches) ++*lc.launches;
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <int MODE, bool NORM>
+cudaError_t launch_mode(const LaunchCtx &lc, const StreamParams &p, int J, int grid, size_t smem) {
+    switch (J) {
+        case 1: return launch_j<1, MODE, NORM>(lc, p, grid, smem);
+        case 2: return launch_j<2, MODE, NORM>(lc, p, grid, smem);
+        case 3: return launch_j<3, MODE, NORM>(lc, p, grid, smem);
+        case 4: return launch_j<4, MODE, NORM>(lc, p, grid, smem);
+        case 5: case 6: return launch_j<6, MODE, NORM>(lc, p, grid, smem);
+        case 7: case 8: return launch_j<8, MODE, NORM>(lc, p, grid, smem);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// Stage geometry for a shape: consumer warps per row, rows per stage.  Measured preferences: stages of 24-52 KB
+// (each is one bulk copy; the per-stage handshake amortises and the copy engine's request rate never binds),
+// an even number of rows per warp per stage (rows are processed in pairs), K slices of 2 KB or more, an even row
+// count per stage when rows pair up as gate/up, and then the best balance over the SMs.
+bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int *ksplit_out, int *rps_out) {
+    double best = -1.0;
+#ifdef NNC_TUNING
+    if (const char *g = getenv("NNC_GEMV_GEOM")) {   // "ksplit,rps": tuning builds only
+        if (sscanf(g, "%d,%d", ksplit_out, rps_out) == 2) return true;
+    }
+#endif
+    const int row_bytes = K * 2;
+    for (int ks = 8; ks >= 1; ks >>= 1) {
+        if (K % (8 * ks)) continue;
+        const int kw = K / ks;
+        if ((kw + 255) / 256 > 8) continue;     // at most 8 chunks per lane
+        if (kw * 2 < 512 && ks > 1) continue;
+        const int gpi = kConsumerWarps / ks;
+        for (int rps = gpi; rps <= kBlockRows; rps += gpi) {
+            if (pairs && (rps & 1)) continue;
+            const long bytes = (long)rps * row_bytes;
+            if (bytes > kRingBytes / 4) break;
+            const int rw = rps / gpi;
+            if (rw > 8) break;
+            const int n_stages = (n_out + rps - 1) / rps;
+            const int grid = n_stages < sm_count ? n_stages : sm_count;
+            const int per = (n_stages + grid - 1) / grid;
+            double score = (double)n_stages / ((double)per * grid);
+            if (rw & 1) score *= 0.85;
+            if (bytes < 8192) score *= 0.80;
+            else if (bytes < 16384) score *= 0.90;
+            else if (bytes < 24576) score *= 0.95;
+            if (kw * 2 < 1024) score *= 0.90;
+            else if (kw * 2 < 2048) score *= 0.93;
+            if (score > best) { best = score; *ksplit_out = ks; *rps_out = rps; }
+        }
+    }
+    return best > 0.0;
+}
+
+}  // namespace
+
+bool gemv_stream_supported(int n_out, int n_in, int mode) {
+    int ks, rps;
+    if (n_out < 1 || n_in % 8 || n_in < 64 || (mode == kGemvSwiglu && n_out % 2)) return false;
+    return pick_geometry(n_out, n_in, 148, mode == kGemvSwiglu, &ks, &rps);
+}
+
+cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
+                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am) {
+    if (!gemv_stream_supported(n_out, n_in, mode)) return cudaErrorInvalidValue;
+    StreamParams p;
+    if (!pick_geometry(n_out, n_in, lc.sm_count, mode == kGemvSwiglu, &p.ksplit, &p.rps)) return cudaErrorInvalidValue;
+    p.W = reinterpret_cast<const uint8_t *>(W);
+    p.x = x; p.y = y; p.gain = gain; p.eps = eps; p.n_out = n_out; p.K = n_in;
+    p.kw = n_in / p.ksplit;
+    const int stage_bytes = p.rps * n_in * 2;
+    int S = kRingBytes / stage_bytes;
+    if (S > kMaxStages) S = kMaxStages;
+    if (S < 2) return cudaErrorInvalidValue;
+    p.stages = S;
+    p.n_stages = (n_out + p.rps - 1) / p.rps;
+    p.pb = kBlockRows / p.rps;
+    if (p.pb < 1) p.pb = 1;
+    p.status = lc.status;
+    p.am = am ? *am : ArgmaxScratch{nullptr, nullptr, nullptr, nullptr};
+    int grid = p.n_stages < lc.sm_count ? p.n_stages : lc.sm_count;
+    if (mode == kGemvLogits && grid > kArgmaxMaxBlocks) grid = kArgmaxMaxBlocks;
+    const size_t smem = (size_t)S * stage_bytes;
+    const int J = (p.kw + 255) / 256;
+    const bool norm = gain != nullptr;
+    switch (mode) {
+        case kGemvStore:
+            return norm ? launch_mode<kGemvStore, true>(lc, p, J, grid, smem) : launch_mode<kGemvStore, false>(lc, p, J, grid, smem);
+        case kGemvResidual:
+            return norm ? launch_mode<kGemvResidual, true>(lc, p, J, grid, smem) : launch_mode<kGemvResidual, false>(lc, p, J, grid, smem);
+        case kGemvSwiglu:
+            return norm ? launch_mode<kGemvSwiglu, true>(lc, p, J, grid, smem) : launch_mode<kGemvSwiglu, false>(lc, p, J, grid, smem);
+        case kGemvLogits:
+            return norm ? launch_mode<kGemvLogits, true>(lc, p, J, grid, smem) : launch_mode<kGemvLogits, false>(lc, p, J, grid, smem);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace nnc

@@ -10,6 +10,7 @@ namespace {
 // x[r][:] = float(E[token_r][:]); one block per row.  Out-of-range ids are clamped.
 __global__ void embed_kernel(const bf16 *__restrict__ E, const int32_t *__restrict__ tokens, float *__restrict__ x,
                              int H, int vocab, float *__restrict__ tap) {
+    NNC_TRACE_SCOPE(1);
     pdl_wait();
     const int r = blockIdx.x;
     int tok = tokens[r];
@@ -37,6 +38,7 @@ qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, 
                            const bf16 *__restrict__ g_k, float eps, const float *__restrict__ rope,
                            bf16 *__restrict__ kcache, bf16 *__restrict__ vcache, int nq, int nkv, int max_seq,
                            const int32_t *__restrict__ d_len, bf16 *__restrict__ q_bf16) {
+    NNC_TRACE_SCOPE(2);
     pdl_wait();
     const int heads = nq + 2 * nkv;
     const int unit = blockIdx.x * 4 + (threadIdx.x >> 5);
@@ -130,6 +132,7 @@ __global__ void copy_f32_kernel(const float *__restrict__ src, float *__restrict
 }
 
 __global__ void add_len_kernel(int32_t *d_len, int delta) {
+    NNC_TRACE_SCOPE(3);
     pdl_wait();
     if (threadIdx.x == 0) *d_len += delta;
 }

@@ -13,6 +13,7 @@
 #include <tuple>
 #include <vector>
 
+#include "common.cuh"
 #include "nnc_internal.h"
 
 using namespace nnc;
@@ -153,7 +154,7 @@ int fail(nnc_model *m, int code, const char *fmt, ...) {
             return fail(m, NNC_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
     } while (0)
 
-LaunchCtx ctx(nnc_model *m, bool pdl) { return LaunchCtx{m->stream, m->sm_count, pdl, &m->launches}; }
+LaunchCtx ctx(nnc_model *m, bool pdl) { return LaunchCtx{m->stream, m->sm_count, pdl, &m->launches, m->d_status}; }
 
 // One decoder layer for a single token (batch 1) on the residual stream m->x.
 int layer_decode_b1(nnc_model *m, int l, const LaunchCtx &lc, int n_splits) {
@@ -162,10 +163,9 @@ int layer_decode_b1(nnc_model *m, int l, const LaunchCtx &lc, int n_splits) {
     bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
     bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
     NNC_CUDA(m, launch_gemv(lc, w.wqkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr));
-    NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkv, 1, 1, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
-                                           c.n_kv_heads, c.max_seq, m->d_len, nullptr));
+    const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
     NNC_CUDA(m, launch_attn_decode(lc, m->qkv, m->qkvd(), kc, vc, m->attn_out, nullptr, nullptr, m->qd(), m->part, m->tickets,
-                                   m->d_len, 1, 1, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits));
+                                   m->d_len, 1, 1, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
     NNC_CUDA(m, launch_gemv(lc, w.wo, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr));
     NNC_CUDA(m, launch_gemv(lc, w.wgu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr));
     NNC_CUDA(m, launch_gemv(lc, w.wd, m->act, m->x, c.hidden, c.intermediate, nullptr, 0.f, kGemvResidual, nullptr));
@@ -201,12 +201,13 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
         bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
         NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_in, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
         NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wqkv, m->qkvt, nullptr, R, qkvd, H, qkvd, kEpiStoreF32, m->d_status));
-        NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
-                                               c.n_kv_heads, c.max_seq, m->d_len, nullptr));
         if (T == 1) {
+            const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
             NNC_CUDA(m, launch_attn_decode(lc, m->qkvt, qkvd, kc, vc, nullptr, m->ob, m->ob_lo, qd, m->part, m->tickets, m->d_len, 1,
-                                           batch, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits));
+                                           batch, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
         } else {
+            NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
+                                                   c.n_kv_heads, c.max_seq, m->d_len, nullptr));
             NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, c.n_q_heads, c.n_kv_heads, c.max_seq, m->d_len));
         }
         NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status));
@@ -570,6 +571,41 @@ const char *nnc_status_string(int status) {
     return "unknown status";
 }
 
+#ifdef NNC_TRACE
+}  // extern "C"
+namespace nnc {
+static std::vector<void (*)(TraceRec *, unsigned *)> &trace_binders() {
+    static std::vector<void (*)(TraceRec *, unsigned *)> v;
+    return v;
+}
+void trace_register(void (*bind)(TraceRec *, unsigned *)) { trace_binders().push_back(bind); }
+static TraceRec *g_trace_dev;
+static unsigned *g_trace_cnt_dev;
+}  // namespace nnc
+extern "C" {
+// tracing builds only.  enable: allocates the record buffer (cudaMalloc -- tracing builds are not the product)
+// and points every translation unit at it.  dump: copies the records out, resets the count, returns it.
+int nnc_trace_enable(void) {
+    if (!nnc::g_trace_dev) {
+        if (cudaMalloc(&nnc::g_trace_dev, sizeof(nnc::TraceRec) * nnc::kTraceMax) != cudaSuccess) return -1;
+        if (cudaMalloc(&nnc::g_trace_cnt_dev, 4) != cudaSuccess) return -1;
+        cudaMemset(nnc::g_trace_cnt_dev, 0, 4);
+    }
+    for (auto b : nnc::trace_binders()) b(nnc::g_trace_dev, nnc::g_trace_cnt_dev);
+    return (int)nnc::trace_binders().size();
+}
+int nnc_trace_dump(void *out, int max_records) {
+    unsigned n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpy(&n, nnc::g_trace_cnt_dev, 4, cudaMemcpyDeviceToHost);
+    if (n > nnc::kTraceMax) n = nnc::kTraceMax;
+    if ((int)n > max_records) n = max_records;
+    if (out && n) cudaMemcpy(out, nnc::g_trace_dev, (size_t)n * sizeof(nnc::TraceRec), cudaMemcpyDeviceToHost);
+    cudaMemset(nnc::g_trace_cnt_dev, 0, 4);
+    return (int)n;
+}
+#endif
+
 // ---- single operations ------------------------------------------------------------------------------
 
 static __device__ int g_op_status;
@@ -578,7 +614,9 @@ static int op_ctx(LaunchCtx &lc, void *stream) {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NNC_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NNC_ERR_CUDA;
-    lc = LaunchCtx{(cudaStream_t)stream, sms, false, nullptr};
+    int *status = nullptr;
+    if (cudaGetSymbolAddress((void **)&status, g_op_status) != cudaSuccess) return NNC_ERR_CUDA;
+    lc = LaunchCtx{(cudaStream_t)stream, sms, false, nullptr, status};
     return NNC_OK;
 }
 
@@ -618,9 +656,12 @@ int nnc_op_status(int32_t *status_out) {
 
 int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t n_in, const void *gain, float eps,
                 int32_t mode, void *cuda_stream) {
+    const bool chained = (mode & NNC_GEMV_CHAINED) != 0;
+    mode &= ~NNC_GEMV_CHAINED;
     if (!W || !x || !y || mode < 0 || mode > 2) return NNC_ERR_INVALID_ARG;
     LaunchCtx lc;
     if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    lc.pdl = chained;
     cudaError_t e = launch_gemv(lc, (const bf16 *)W, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
@@ -646,9 +687,9 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
     float *part = (float *)scratch;
     uint32_t *tickets = (uint32_t *)((char *)scratch + (attn_decode_scratch_floats(batch, n_q_heads, kAttnMaxSplits) * 4 + 255) / 256 * 256);
     if (cudaMemsetAsync(tickets, 0, (size_t)batch * n_kv_heads * 4, lc.stream) != cudaSuccess) return NNC_ERR_CUDA;
-    cudaError_t e = launch_attn_decode(lc, q, n_q_heads * 128, (const bf16 *)kcache, (const bf16 *)vcache, out, nullptr, nullptr,
-                                       n_q_heads * 128, part, tickets, nullptr, n_ctx, batch, n_q_heads, n_kv_heads,
-                                       max_seq, n_splits);
+    cudaError_t e = launch_attn_decode(lc, q, n_q_heads * 128, (bf16 *)const_cast<void *>(kcache), (bf16 *)const_cast<void *>(vcache),
+                                       out, nullptr, nullptr, n_q_heads * 128, part, tickets, nullptr, n_ctx, batch, n_q_heads,
+                                       n_kv_heads, max_seq, n_splits, nullptr);
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 

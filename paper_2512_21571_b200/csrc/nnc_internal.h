@@ -15,6 +15,7 @@ struct LaunchCtx {
     int sm_count;
     bool pdl;           // launch with programmatic stream serialization (kernels call pdl_wait themselves)
     int64_t *launches;  // bumped once per kernel launch (may be null)
+    int *status;        // device status word raised by kernels whose bounded waits run out (may be null)
 };
 
 template <typename... KArgs, typename... Args>
@@ -46,6 +47,12 @@ struct ArgmaxScratch {
 cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
                         const bf16 *gain, float eps, int mode, const ArgmaxScratch *am);
 
+// streaming form (decode_gemv_stream.cu): n_in a multiple of 8 up to 16384 (8192 for SwiGLU); launch_gemv uses it
+// whenever the shape allows and falls back to the plain-load kernel otherwise
+bool gemv_stream_supported(int n_out, int n_in, int mode);
+cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
+                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am);
+
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
                          int vocab, float *tap);
@@ -62,10 +69,18 @@ cudaError_t launch_add_len(const LaunchCtx &lc, int32_t *d_len, int delta);
 constexpr int kAttnMaxSplits = 64;
 int attn_decode_splits(int sm_count, int batch, int nkv, int max_ctx);
 size_t attn_decode_scratch_floats(int batch, int nq, int n_splits);
-cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, const bf16 *kcache,
-                               const bf16 *vcache, float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride,
-                               float *part, uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
-                               int max_seq, int n_splits);
+// fused != null: q points at the raw fused QKV activation of the new token (query heads, then key heads, then
+// value heads); the kernel applies the per-head RMSNorm + RoPE to q and k itself and appends the bf16 K/V row
+// at position *d_len + len_add - 1 before attending to it.
+struct AttnFused {
+    const bf16 *g_q, *g_k;
+    const float *rope;
+    float eps;
+};
+cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_stride, bf16 *kcache, bf16 *vcache,
+                               float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride, float *part,
+                               uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
+                               int max_seq, int n_splits, const AttnFused *fused);
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
                                 const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
                                 const int32_t *d_len);
