@@ -22,7 +22,7 @@ namespace nnc {
 
 namespace {
 
-constexpr int kPartStride = kHeadDim + 2;  // o~[128], m, l
+constexpr int kPartStride = kHeadDim + 4;  // o~[128], m, l, 2 pad words (rows stay 16-byte aligned)
 constexpr int kWarps = 4;
 
 __device__ __forceinline__ uint4 ldg_cg(const void *p) {
@@ -124,6 +124,31 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(const AttnPara
     const int n_active = (n_ctx + chunk - 1) / chunk;
     if (c0 >= n_ctx) return;  // whole CTA; takes no ticket (n_active counts only non-empty ranges)
 
+    // ---- K/V fragment loads of one block of 16 positions: K rows p0 + 8h + g8 (h = 0, 1), V rows
+    //      p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9}; rows past the range are clamped here and masked later ----
+    uint4 kf[2][4], vf[4][2];
+    auto load_block = [&](int p0) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int pos = min(p0 + 8 * h + g8, c1 - 1);
+            const bf16 *kr = kbase + (size_t)pos * kHeadDim + 8 * t4;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) kf[h][c] = ldg_cg(kr + 32 * c);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int pos = min(p0 + 2 * t4 + (r & 1) + 8 * (r >> 1), c1 - 1);
+            const bf16 *vr = vbase + (size_t)pos * kHeadDim + 8 * g8;
+            vf[r][0] = ldg_cg(vr);
+            vf[r][1] = ldg_cg(vr + 64);
+        }
+    };
+    const int n_blocks = (c1 - c0 + 15) >> 4;
+    // the warp's first block is requested now and lands while the queries are prepared -- unless it holds the row
+    // that is appended below
+    const bool early = warp < n_blocks && !(FUSED && c0 + warp * 16 + 16 >= n_ctx);
+    if (early) load_block(c0 + warp * 16);
+
     // ---- queries (and, fused, the new token's K/V row) ----
     const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);   // scores in log2 units
     const float *qrow = p.q + (size_t)b * p.q_row_stride;
@@ -178,25 +203,9 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(const AttnPara
     for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run = -INFINITY, l_run = 0.f;   // per row g8 (identical across the 4 lanes of a row); l is a per-lane partial
 
-    const int n_blocks = (c1 - c0 + 15) >> 4;
     for (int blk = warp; blk < n_blocks; blk += kWarps) {
         const int p0 = c0 + blk * 16;
-        // ---- loads: K rows p0 + 8h + g8 (h = 0, 1), V rows p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9} ----
-        uint4 kf[2][4], vf[4][2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int pos = min(p0 + 8 * h + g8, c1 - 1);   // rows past the range are clamped and masked below
-            const bf16 *kr = kbase + (size_t)pos * kHeadDim + 8 * t4;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) kf[h][c] = ldg_cg(kr + 32 * c);
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int pos = min(p0 + 2 * t4 + (r & 1) + 8 * (r >> 1), c1 - 1);
-            const bf16 *vr = vbase + (size_t)pos * kHeadDim + 8 * g8;
-            vf[r][0] = ldg_cg(vr);
-            vf[r][1] = ldg_cg(vr + 64);
-        }
+        if (!(early && blk == warp)) load_block(p0);
         // ---- scores: S[h] = Q K^T for the 8 positions of half h ----
         float s[2][4];
 #pragma unroll
@@ -317,30 +326,33 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(const AttnPara
         if (lane == 0) inv_l[g] = 1.f / L;
     }
     __syncthreads();
-    float acc[G];
+    // one warp per head, 4 output elements per lane: 16-byte loads, a batch of splits in flight at once
+    for (int g = warp; g < G; g += kWarps) {
+        const float *pp = pbase + (size_t)g * p.n_splits * kPartStride + 4 * lane;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int cb = 0; cb < n_active; cb += 24) {
+            float4 v[24];
 #pragma unroll
-    for (int g = 0; g < G; ++g) acc[g] = 0.f;
-    for (int cb = 0; cb < n_active; cb += 8) {
-        float v[G][8];
+            for (int u = 0; u < 24; ++u)
+                v[u] = (cb + u < n_active) ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(cb + u) * kPartStride))
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-                v[g][u] = (cb + u < n_active) ? __ldcg(pbase + ((size_t)g * p.n_splits + cb + u) * kPartStride + tid) : 0.f;
-#pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int u = 0; u < 8; ++u) acc[g] = fmaf(cb + u < n_active ? wgt[g][cb + u] : 0.f, v[g][u], acc[g]);
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-        const float r = acc[g] * inv_l[g];
-        const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + tid;
-        if (p.out_f32) p.out_f32[oi] = r;
+            for (int u = 0; u < 24; ++u) {
+                const float w = (cb + u < n_active) ? wgt[g][cb + u] : 0.f;
+                acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+                acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+            }
+        }
+        const float il = inv_l[g];
+        const float4 r = make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il);
+        const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + 4 * lane;
+        if (p.out_f32) *reinterpret_cast<float4 *>(p.out_f32 + oi) = r;
         if (p.out_bf16) {
-            const bf16 hi = __float2bfloat16_rn(r);
-            p.out_bf16[oi] = hi;
-            if (p.out_bf16_lo) p.out_bf16_lo[oi] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            const uint2 hi = make_uint2(pack_bf16x2(r.x, r.y), pack_bf16x2(r.z, r.w));
+            *reinterpret_cast<uint2 *>(p.out_bf16 + oi) = hi;
+            if (p.out_bf16_lo)
+                *reinterpret_cast<uint2 *>(p.out_bf16_lo + oi) =
+                    make_uint2(pack_bf16x2(r.x - bf16_lo(hi.x), r.y - bf16_hi(hi.x)), pack_bf16x2(r.z - bf16_lo(hi.y), r.w - bf16_hi(hi.y)));
         }
     }
     if (tid == 0) p.tickets[b * p.nkv + j] = 0u;

@@ -243,8 +243,8 @@ cudaError_t launch_rows(const LaunchCtx &lc, const bf16 *W, const float *x, floa
 }  // namespace
 
 cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                        const bf16 *gain, float eps, int mode, const ArgmaxScratch *am) {
-    if (gemv_stream_supported(n_out, n_in, mode)) return launch_gemv_stream(lc, W, x, y, n_out, n_in, gain, eps, mode, am);
+                        const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr) {
+    if (gemv_stream_supported(n_out, n_in, mode)) return launch_gemv_stream(lc, W, x, y, n_out, n_in, gain, eps, mode, am, ctr);
     if (n_in % 8 != 0 || n_in <= 0 || n_out <= 0 || (size_t)n_in * 4 > 200 * 1024) return cudaErrorInvalidValue;
     ArgmaxScratch a = am ? *am : ArgmaxScratch{nullptr, nullptr, nullptr, nullptr};
     const bool norm = gain != nullptr;

@@ -5,10 +5,12 @@
 //     keeps the ring full with cp.async.bulk copies (the 1-D form of TMA) of 8-32 KB each -- whole consecutive
 //     rows, which are contiguous in the row-major matrix -- so ~100 KB per SM are outstanding without holding
 //     registers, and each copy is large enough that the copy engine's request rate is not the limit;
-//   - the matrix is cut into stages of `rps` rows and every CTA takes an equal contiguous run of stages
-//     (~14 or more per SM whatever the shape: no wave quantisation);
+//   - the matrix is cut into stages of `rps` rows; CTAs claim short runs of consecutive stages from a global
+//     counter (first run fixed, later runs by atomic, claimed one run ahead), so there is no wave quantisation
+//     and SMs that stream faster take more of the matrix;
 //   - inside a stage `ksplit` warps share a row, each taking a contiguous K slice whose activations it holds in
-//     registers (optionally RMS-normalised on the way in), so shared memory carries weights only;
+//     registers (times the norm gain when the RMSNorm prologue is fused; the scalar 1/rms is applied to the
+//     finished sums), so shared memory carries weights only;
 //   - per-row partial sums meet in a small double-buffered shared array and are folded in fixed order every
 //     ~64 rows (deterministic: no float atomics), where the epilogue runs: store, residual add, SwiGLU on
 //     interleaved gate/up rows, or logits + arg-max candidates (the last CTA folds those; nobody waits);
@@ -102,6 +104,8 @@ struct StreamParams {
     int stages;    // ring depth
     int n_stages;  // stages in the whole matrix = ceil(n_out / rps)
     int pb;        // stages per fold block = kBlockRows / rps (at least 1)
+    int claim;     // consecutive stages per work claim
+    uint32_t *ctr; // {next run, CTAs done}: zero between launches; null = runs are dealt round-robin
     int *status;   // raised if a bounded wait runs out
     ArgmaxScratch am;
 };
@@ -113,6 +117,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ __align__(8) uint64_t full[kMaxStages], empty[kMaxStages];
     __shared__ float part[2][kBlockRows][kConsumerWarps];
+    __shared__ int slot_row[kMaxStages];        // first row of the stage held by each ring slot (-1: end of work)
+    __shared__ int blk_row[2][kBlockRows];      // first row of each stage of the current fold block
+    __shared__ float ssq[kConsumerWarps];       // sum of squares of each warp's activation slice
     __shared__ float red[kConsumerWarps];
     __shared__ int red_i[kConsumerWarps];
     __shared__ bool is_last;
@@ -121,10 +128,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     const int S = p.stages;
     const uint32_t row_bytes = (uint32_t)p.K * 2u;
     const uint32_t stage_bytes = (uint32_t)p.rps * row_bytes;
-
-    const int per = p.n_stages / gridDim.x, rem = p.n_stages % gridDim.x;
-    const int st0 = blockIdx.x * per + min((int)blockIdx.x, rem);
-    const int n_st = per + ((int)blockIdx.x < rem ? 1 : 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -137,21 +140,44 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     pdl_launch_dependents();
 
     if (warp == kConsumerWarps) {
-        // ---------------- producer: streams this CTA's stages; never waits on the previous kernel ----------------
+        // ---------------- producer: streams stages into the ring; never waits on the previous kernel ----------------
+        // Work is claimed in runs of `claim` consecutive stages.  Each CTA starts with a fixed share that fills its ring
+        // (runs i, i + grid, ...); later runs come from a global counter, so SMs that stream faster (they do differ
+        // by ~15 %) simply take more.
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int s = 0; s < n_st; ++s) {
-                if (!mbar_wait_bounded(smem_u32(&empty[stage]), phase ^ 1u)) {
-                    if (p.status) atomicExch(p.status, 17);
-                    break;
+            bool ok = true;
+            const int n_runs = (p.n_stages + p.claim - 1) / p.claim;
+            const int n_static = (S + p.claim - 1) / p.claim;
+            const int grid = (int)gridDim.x;
+            // run number of this CTA's k-th claim; claims are issued three runs ahead of the copies
+            auto claim_id = [&](int k) {
+                return (k < n_static || !p.ctr) ? (int)blockIdx.x + k * grid : grid * n_static + (int)atomicAdd(p.ctr, 1u);
+            };
+            int r0 = claim_id(0), r1 = claim_id(1), r2 = claim_id(2);
+            for (int k = 3; r0 < n_runs && ok; ++k) {
+                const int r3 = claim_id(k);
+                const int s_end = min((r0 + 1) * p.claim, p.n_stages);
+                for (int s = r0 * p.claim; s < s_end; ++s) {
+                    if (!mbar_wait_bounded(smem_u32(&empty[stage]), phase ^ 1u)) { ok = false; break; }
+                    const int row0 = s * p.rps;
+                    const int rows = min(p.rps, p.n_out - row0);
+                    slot_row[stage] = row0;
+                    bulk_load(smem_u32(ring) + (uint32_t)stage * stage_bytes, p.W + (size_t)row0 * row_bytes,
+                              (uint32_t)rows * row_bytes, smem_u32(&full[stage]));
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
-                const int row0 = (st0 + s) * p.rps;
-                const int rows = min(p.rps, p.n_out - row0);
-                bulk_load(smem_u32(ring) + (uint32_t)stage * stage_bytes, p.W + (size_t)row0 * row_bytes,
-                          (uint32_t)rows * row_bytes, smem_u32(&full[stage]));
-                if (++stage == S) { stage = 0; phase ^= 1u; }
+                r0 = r1; r1 = r2; r2 = r3;
             }
+            if (ok && mbar_wait_bounded(smem_u32(&empty[stage]), phase ^ 1u)) {
+                slot_row[stage] = -1;   // end of work for this CTA
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[stage])) : "memory");
+            } else if (p.status) {
+                atomicExch(p.status, 17);
+            }
+            // the CTA that stops claiming last puts the counters back to zero for the next launch of this call site
+            if (p.ctr && atomicAdd(p.ctr + 1, 1u) == gridDim.x - 1) { p.ctr[0] = 0u; p.ctr[1] = 0u; }
         }
         return;
     }
@@ -172,7 +198,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     pdl_wait();
     NNC_TRACE_MARK();
 
-    // this warp's activation slice, in registers
+    // this warp's activation slice, in registers.  With the norm prologue it holds x * gain; the scalar
+    // 1/rms(x) is applied to the finished row sums at the fold, so nothing waits for the sum of squares.
     float xr[J][8];
     float ss = 0.f;
 #pragma unroll
@@ -190,55 +217,47 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
         if (NORM) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
+            const uint4 g = gr[i];
+            xr[i][0] *= bf16_lo(g.x); xr[i][1] *= bf16_hi(g.x);
+            xr[i][2] *= bf16_lo(g.y); xr[i][3] *= bf16_hi(g.y);
+            xr[i][4] *= bf16_lo(g.z); xr[i][5] *= bf16_hi(g.z);
+            xr[i][6] *= bf16_lo(g.w); xr[i][7] *= bf16_hi(g.w);
         }
     }
     if (NORM) {
         ss = warp_sum(ss);
-        if (lane == 0) red[warp] = ss;
-        consumer_sync();
-        float tot = 0.f;
-        for (int k = 0; k < ksplit; ++k) tot += red[k];   // warps 0 .. ksplit-1 hold the ksplit distinct slices
-        const float inv = rsqrtf(tot / (float)p.K + p.eps);
-#pragma unroll
-        for (int i = 0; i < J; ++i) {
-            const int c = lane + 32 * i;
-            {
-                const uint4 g = gr[i];
-                xr[i][0] *= inv * bf16_lo(g.x); xr[i][1] *= inv * bf16_hi(g.x);
-                xr[i][2] *= inv * bf16_lo(g.y); xr[i][3] *= inv * bf16_hi(g.y);
-                xr[i][4] *= inv * bf16_lo(g.z); xr[i][5] *= inv * bf16_hi(g.z);
-                xr[i][6] *= inv * bf16_lo(g.w); xr[i][7] *= inv * bf16_hi(g.w);
-            }
-        }
-        consumer_sync();   // red is reused by the arg-max fold
+        if (lane == 0) ssq[warp] = ss;   // read after the first consumer_sync below
     }
 
     float best_v = -INFINITY;
     int best_i = 0x7fffffff;
     int stage = 0;
     uint32_t phase = 0;
-    bool ok = true;
+    bool ok = true, done = false;
+    float inv = 1.f;
     const uint32_t slice_off = (uint32_t)ks * (uint32_t)p.kw * 2u;
+    const int t = threadIdx.x;
+    const int fold_unit = (MODE == kGemvSwiglu) ? (p.rps >> 1) : p.rps;   // outputs per stage
+    const int tj = t / fold_unit, tr = t % fold_unit;                      // this thread's (stage in block, output in stage)
 
-    for (int b0 = 0, blk = 0; b0 < n_st; b0 += p.pb, ++blk) {
-        const int nb = min(p.pb, n_st - b0);
+    for (int blk = 0; !done; ++blk) {
         const int buf = blk & 1;
-        const int block_row0 = (st0 + b0) * p.rps;
-        const int rows_here = min(nb * p.rps, p.n_out - block_row0);
-        float y_old = 0.f;   // residual mode: fetched now, used at the fold (hides the global-load latency)
-        if (MODE == kGemvResidual && (int)threadIdx.x < rows_here) y_old = p.y[block_row0 + threadIdx.x];
-        for (int j = 0; j < nb; ++j) {
-            if (ok && !mbar_wait_bounded(smem_u32(&full[stage]), phase)) {
-                ok = false;
+        int nb = 0;
+        for (int j = 0; j < p.pb; ++j) {
+            if (!mbar_wait_bounded(smem_u32(&full[stage]), phase)) {
+                ok = false; done = true;
                 if (lane == 0 && p.status) atomicExch(p.status, 16);
+                break;
             }
+            const int row0 = slot_row[stage];
+            if (row0 < 0) { done = true; break; }
+            if (t == 0) blk_row[buf][j] = row0;
             const uint32_t sbase = smem_u32(ring) + (uint32_t)stage * stage_bytes + slice_off;
             // rows of this stage owned by the warp, two at a time (independent load / FMA streams, one joint reduction)
-            for (int m = 0; m < rw && ok; m += 2) {
+            for (int m = 0; m < rw; m += 2) {
                 const int r_in_stage = gi + gpi * m;
-                const int r_in_block = j * p.rps + r_in_stage;
-                if (block_row0 + r_in_block >= p.n_out) break;   // ragged last stage (warp-uniform)
-                const bool two = (m + 1 < rw) && (block_row0 + r_in_block + gpi < p.n_out);
+                if (row0 + r_in_stage >= p.n_out) break;   // ragged last stage (warp-uniform)
+                const bool two = (m + 1 < rw) && (row0 + r_in_stage + gpi < p.n_out);
                 const uint32_t rbase0 = sbase + (uint32_t)r_in_stage * row_bytes;
                 const uint32_t rbase1 = two ? rbase0 + (uint32_t)gpi * row_bytes : rbase0;
                 uint4 w0[J], w1[J];
@@ -259,29 +278,43 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
                 keep += __shfl_xor_sync(0xffffffffu, upper ? s0 : s1, 16);
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) keep += __shfl_xor_sync(0xffffffffu, keep, o);
+                const int r_in_block = j * p.rps + r_in_stage;
                 if (lane == 0) part[buf][r_in_block][ks] = keep;
                 if (lane == 16 && two) part[buf][r_in_block + gpi][ks] = keep;
             }
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[stage])) : "memory");
             if (++stage == S) { stage = 0; phase ^= 1u; }
+            ++nb;
         }
         consumer_sync();
+        if (NORM && blk == 0) {
+            float tot = 0.f;
+            for (int k = 0; k < ksplit; ++k) tot += ssq[k];   // warps 0 .. ksplit-1 hold the ksplit distinct slices
+            inv = rsqrtf(tot / (float)p.K + p.eps);
+        }
         // ---- fold the ksplit partial sums of each row in fixed order; epilogue ----
-        const int t = threadIdx.x;
-        if (MODE == kGemvSwiglu) {
-            if (2 * t + 1 < rows_here) {
-                float g = 0.f, u = 0.f;
-                for (int k = 0; k < ksplit; ++k) { g += part[buf][2 * t][k]; u += part[buf][2 * t + 1][k]; }
-                p.y[(block_row0 >> 1) + t] = g / (1.f + __expf(-g)) * u;
+        if (tj < nb) {
+            const int row0 = blk_row[buf][tj];
+            if (MODE == kGemvSwiglu) {
+                const int r = tj * p.rps + 2 * tr;
+                if (row0 + 2 * tr + 1 < p.n_out) {
+                    float g = 0.f, u = 0.f;
+                    for (int k = 0; k < ksplit; ++k) { g += part[buf][r][k]; u += part[buf][r + 1][k]; }
+                    g *= inv; u *= inv;
+                    p.y[(row0 >> 1) + tr] = g / (1.f + __expf(-g)) * u;
+                }
+            } else if (row0 + tr < p.n_out) {
+                float v = 0.f;
+                for (int k = 0; k < ksplit; ++k) v += part[buf][tj * p.rps + tr][k];
+                v *= inv;
+                const int row = row0 + tr;
+                // residual: each element is touched by exactly one thread of one CTA per launch, so a reduction
+                // without return value gives the same sum as load-add-store and exposes no load latency
+                if (MODE == kGemvResidual) atomicAdd(p.y + row, v);
+                else p.y[row] = v;
+                if (MODE == kGemvLogits && better(v, row, best_v, best_i)) { best_v = v; best_i = row; }
             }
-        } else if (t < rows_here) {
-            float v = 0.f;
-            for (int k = 0; k < ksplit; ++k) v += part[buf][t][k];
-            const int row = block_row0 + t;
-            if (MODE == kGemvResidual) v += y_old;
-            p.y[row] = v;
-            if (MODE == kGemvLogits && better(v, row, best_v, best_i)) { best_v = v; best_i = row; }
         }
     }
 
@@ -421,7 +454,7 @@ bool gemv_stream_supported(int n_out, int n_in, int mode) {
 }
 
 cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am) {
+                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr) {
     if (!gemv_stream_supported(n_out, n_in, mode)) return cudaErrorInvalidValue;
     StreamParams p;
     if (!pick_geometry(n_out, n_in, lc.sm_count, mode == kGemvSwiglu, &p.ksplit, &p.rps)) return cudaErrorInvalidValue;
@@ -438,7 +471,13 @@ cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *
     if (p.pb < 1) p.pb = 1;
     p.status = lc.status;
     p.am = am ? *am : ArgmaxScratch{nullptr, nullptr, nullptr, nullptr};
-    int grid = p.n_stages < lc.sm_count ? p.n_stages : lc.sm_count;
+    // claims of ~64 KB keep each CTA's reads in longer sequential pieces (measured: better on large matrices);
+    // matrices with few stages per SM claim stage by stage so that the tail stays short
+    p.claim = (stage_bytes >= 49152 || p.n_stages < 16 * lc.sm_count) ? 1 : (65536 + stage_bytes - 1) / stage_bytes;
+    if (stage_bytes < 16384 && p.claim == 1) p.claim = (32768 + stage_bytes - 1) / stage_bytes;
+    p.ctr = ctr;
+    const int n_runs = (p.n_stages + p.claim - 1) / p.claim;
+    int grid = n_runs < lc.sm_count ? n_runs : lc.sm_count;
     if (mode == kGemvLogits && grid > kArgmaxMaxBlocks) grid = kArgmaxMaxBlocks;
     const size_t smem = (size_t)S * stage_bytes;
     const int J = (p.kw + 255) / 256;

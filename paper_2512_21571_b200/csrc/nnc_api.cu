@@ -32,7 +32,7 @@ struct Plan {
     // offsets
     std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
-    size_t x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
+    size_t gemv_ctr, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
     size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
     size_t take(size_t bytes) {
         const size_t o = total;
@@ -75,6 +75,7 @@ void make_plan(const nnc_config &c, Plan &p) {
     p.kcache = p.take(kv);
     p.vcache = p.take(kv);
     p.rope = p.take((size_t)c.max_seq * 128 * 4);
+    p.gemv_ctr = p.take(((size_t)c.n_layers * 4 + 2) * 16);
     p.x = p.take(H * 4);
     p.qkv = p.take(qkvd * 4);
     p.attn_out = p.take(qd * 4);
@@ -112,6 +113,7 @@ struct nnc_model {
     bf16 *embed, *lm_head, *g_final, *kcache, *vcache;
     float *rope, *x, *qkv, *attn_out, *act, *part;
     uint32_t *tickets;
+    uint32_t *gemv_ctr;  // 4 words per GEMV call site (4 per layer + lm_head): dynamic work counters, zero at rest
     ArgmaxScratch am;
     int32_t *d_len, *d_status, *d_tokens, *d_argmax;
     float *xt, *qkvt, *logits_stage;
@@ -162,13 +164,14 @@ int layer_decode_b1(nnc_model *m, int l, const LaunchCtx &lc, int n_splits) {
     const LayerW &w = m->layers[l];
     bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
     bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
-    NNC_CUDA(m, launch_gemv(lc, w.wqkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr));
+    uint32_t *ctr = m->gemv_ctr + (size_t)l * 16;
+    NNC_CUDA(m, launch_gemv(lc, w.wqkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr, ctr));
     const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
     NNC_CUDA(m, launch_attn_decode(lc, m->qkv, m->qkvd(), kc, vc, m->attn_out, nullptr, nullptr, m->qd(), m->part, m->tickets,
                                    m->d_len, 1, 1, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
-    NNC_CUDA(m, launch_gemv(lc, w.wo, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr));
-    NNC_CUDA(m, launch_gemv(lc, w.wgu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr));
-    NNC_CUDA(m, launch_gemv(lc, w.wd, m->act, m->x, c.hidden, c.intermediate, nullptr, 0.f, kGemvResidual, nullptr));
+    NNC_CUDA(m, launch_gemv(lc, w.wo, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr, ctr + 4));
+    NNC_CUDA(m, launch_gemv(lc, w.wgu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr, ctr + 8));
+    NNC_CUDA(m, launch_gemv(lc, w.wd, m->act, m->x, c.hidden, c.intermediate, nullptr, 0.f, kGemvResidual, nullptr, ctr + 12));
     return NNC_OK;
 }
 
@@ -183,7 +186,8 @@ int decode_b1_launches(nnc_model *m, const int32_t *tokens, float *logits, int32
     }
     ArgmaxScratch am = m->am;
     am.out = argmax;
-    NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->x, logits, c.vocab, c.hidden, m->g_final, c.rms_eps, kGemvLogits, &am));
+    NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->x, logits, c.vocab, c.hidden, m->g_final, c.rms_eps, kGemvLogits, &am,
+                            m->gemv_ctr + (size_t)c.n_layers * 16));
     NNC_CUDA(m, launch_add_len(lc, m->d_len, 1));
     return NNC_OK;
 }
@@ -298,6 +302,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         m->kcache = (bf16 *)at(p.kcache); m->vcache = (bf16 *)at(p.vcache); m->rope = (float *)at(p.rope);
         m->x = (float *)at(p.x); m->qkv = (float *)at(p.qkv); m->attn_out = (float *)at(p.attn_out);
         m->act = (float *)at(p.act); m->part = (float *)at(p.part); m->tickets = (uint32_t *)at(p.tickets);
+        m->gemv_ctr = (uint32_t *)at(p.gemv_ctr);
         m->am = ArgmaxScratch{(float *)at(p.am_val), (int32_t *)at(p.am_idx), (uint32_t *)at(p.am_ticket), nullptr};
         m->d_len = (int32_t *)at(p.d_len); m->d_status = (int32_t *)at(p.d_status);
         m->d_tokens = (int32_t *)at(p.d_tokens); m->d_argmax = (int32_t *)at(p.d_argmax);
@@ -352,6 +357,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         }
         NNC_CUDA(m, cudaMemsetAsync(m->tickets, 0, (size_t)c.max_batch * c.n_kv_heads * 4, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->am.ticket, 0, 4, m->stream));
+        NNC_CUDA(m, cudaMemsetAsync(m->gemv_ctr, 0, ((size_t)c.n_layers * 4 + 2) * 16, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->d_len, 0, 4, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->d_status, 0, 4, m->stream));
         NNC_CUDA(m, cudaStreamSynchronize(m->stream));
@@ -609,6 +615,7 @@ int nnc_trace_dump(void *out, int max_records) {
 // ---- single operations ------------------------------------------------------------------------------
 
 static __device__ int g_op_status;
+static __device__ uint32_t g_op_gemv_ctr[8][4];   // work counters of the last 8 nnc_op_gemv calls, used in rotation
 
 static int op_ctx(LaunchCtx &lc, void *stream) {
     int dev = 0, sms = 0;
@@ -662,7 +669,11 @@ int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t 
     LaunchCtx lc;
     if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
     lc.pdl = chained;
-    cudaError_t e = launch_gemv(lc, (const bf16 *)W, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr);
+    uint32_t *ctrs = nullptr;
+    if (cudaGetSymbolAddress((void **)&ctrs, g_op_gemv_ctr) != cudaSuccess) return NNC_ERR_CUDA;
+    static unsigned rotation = 0;
+    cudaError_t e = launch_gemv(lc, (const bf16 *)W, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr,
+                                ctrs + 4 * (rotation++ % 8));
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }

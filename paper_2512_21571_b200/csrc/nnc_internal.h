@@ -44,14 +44,16 @@ struct ArgmaxScratch {
     int32_t *out;       // result; null = no arg-max
 };
 
+// ctr (nullable): two zeroed words owned by this call site, used by the streaming form to hand out work
+// dynamically; a call site may be launched again only after ~4 later GEMVs of the same stream have started.
 cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                        const bf16 *gain, float eps, int mode, const ArgmaxScratch *am);
+                        const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr = nullptr);
 
 // streaming form (decode_gemv_stream.cu): n_in a multiple of 8 up to 16384 (8192 for SwiGLU); launch_gemv uses it
 // whenever the shape allows and falls back to the plain-load kernel otherwise
 bool gemv_stream_supported(int n_out, int n_in, int mode);
 cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am);
+                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr);
 
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
