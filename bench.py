@@ -284,6 +284,9 @@ def kernel_roofline_gemv(shape, peaks, w):
     n_mats = min(shape.n_layers, 12)
     mats = []
     for l in range(n_mats):
+        if w is None:   # --kernel-only: no model was built; any seeded matrix of the shape will do
+            mats.append(synth.normal(9, 100 + l, (2 * I, H), 0.02, torch.bfloat16, "cuda"))
+            continue
         lw = w["layers"][l]
         wgu = torch.empty(2 * I, H, dtype=torch.bfloat16, device="cuda")
         wgu[0::2] = lw["w_gate"]
@@ -311,7 +314,10 @@ def kernel_roofline_gemv(shape, peaks, w):
     return {"bound": "hbm", "kernel": "gemv_stream_kernel<SwiGLU, norm prologue>", "shape": [2 * I, H],
             "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
             "peak_source": peaks["source"], "bytes_per_launch": nbytes, "us_per_launch": round(us, 2),
-            "launches_timed": n, "traffic": None}
+            "launches_timed": n,
+            # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/gemv_stream_kernel_gateup_qwen3-8b.md);
+            # valid for the 24576 x 4096 shape only
+            "traffic": 205.3e6 if (2 * I, H) == (24576, 4096) else None}
 
 
 def kernel_roofline_gemm(shape, peaks, T):
@@ -457,6 +463,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the isolated-kernel and prompt-phase extras")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="time only the dominant kernel of the workload on ~2.4 GB of operands (small enough for a "
+                         "multi-pass profiler capture) and print its roofline object")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     if args.steps is None:
@@ -474,6 +483,14 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
     rank, world = dist_setup(args.gpus)
     peaks = load_peaks()
+    if args.kernel_only:
+        shape = synth.SHAPES[wl["shape"]]
+        if wl["kind"] == "decode" and wl["batch"] == 1:
+            roof = kernel_roofline_gemv(shape, peaks, None)
+        else:
+            roof = kernel_roofline_gemm(shape, peaks, max(wl["batch"] * wl.get("tokens", 1), 32))
+        print(json.dumps({"kernel_only": True, "config": config_of(wl), "roofline": roof}), flush=True)
+        return
     m, shape, w = build_model(wl)
     steps, warmup = args.steps, args.warmup
 
