@@ -1,9 +1,15 @@
-// Causal attention for a block of new tokens (the prompt phase): query at position p attends to cache
+// Causal attention for a block of new tokens (the prompt phase): the query at position p attends to cache
 // positions 0..p of its sequence.  K and V are read from the bf16 cache, which already holds the new tokens.
 //
-// One warp per (token row, query head).  Keys are taken 32 at a time, one per lane for the score (the query
-// sits in shared memory and is broadcast), then the 32 probabilities are shuffled around while every lane
-// accumulates its 4 output elements.  Online softmax in fp32.
+// Flash-attention on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 accumulate):
+//   - grid (query tiles of 128 positions, query heads, sequences), 8 warps; a warp owns 16 query rows and keeps
+//     its Q fragments, the running (m, l) and the 16 x 128 output accumulator in registers;
+//   - K/V tiles of 64 cache positions are staged in shared memory with cp.async (16 bytes per thread, XOR-swizzled
+//     chunks so that ldmatrix is conflict-free), double-buffered: the next tile streams in while the current one
+//     is multiplied.  The G query heads that share a KV head run in different CTAs and meet in L2;
+//   - Q and the probabilities are fed as two bf16 terms each (value + rounding residual), so the products keep
+//     fp32-level accuracy (a single bf16 term costs ~2^-9 per operand, which the parity bar does not allow);
+//   - only the tiles on the diagonal apply the causal mask; query tiles are issued longest first.
 #include "common.cuh"
 #include "nnc_internal.h"
 
@@ -11,77 +17,211 @@ namespace nnc {
 
 namespace {
 
-__global__ void __launch_bounds__(128)
-attn_prefill_kernel(const float *__restrict__ qkv, int rows, int rows_per_seq, const bf16 *__restrict__ kcache,
+constexpr int kBM = 128;   // query rows per CTA
+constexpr int kBN = 64;    // cache positions per tile
+constexpr int kPfWarps = 8;
+constexpr int kTileBytes = kBN * kHeadDim * 2;   // 16 KB
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// value + residual bf16 pairs of two floats
+__device__ __forceinline__ void split_pair(float x, float y, uint32_t &hi, uint32_t &lo) {
+    hi = pack_bf16x2(x, y);
+    lo = pack_bf16x2(x - bf16_lo(hi), y - bf16_hi(hi));
+}
+
+// byte offset of 16-byte chunk `chunk` (0..15) of row `row` inside a [kBN][128] bf16 tile, XOR-swizzled
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+    return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4));
+}
+
+// cp.async of one K and one V tile (cache positions k0 .. k0 + 63, clamped to the last valid row) into a stage
+__device__ __forceinline__ void load_tile(uint32_t stage_base, const bf16 *kbase, const bf16 *vbase, int k0, int last_row,
+                                          int tid) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = tid + 256 * i;          // 1024 chunks of 16 bytes per tile
+        const int row = idx >> 4, chunk = idx & 15;
+        const size_t src = (size_t)min(k0 + row, last_row) * kHeadDim + chunk * 8;
+        cp_async16(stage_base + tile_off(row, chunk), kbase + src);
+        cp_async16(stage_base + kTileBytes + tile_off(row, chunk), vbase + src);
+    }
+}
+
+__global__ void __launch_bounds__(kPfWarps * 32, 1)
+attn_prefill_kernel(const float *__restrict__ qkv, int rows_per_seq, const bf16 *__restrict__ kcache,
                     const bf16 *__restrict__ vcache, bf16 *__restrict__ out, bf16 *__restrict__ out_lo, int nq, int nkv,
                     int max_seq, const int32_t *__restrict__ d_len) {
-    __shared__ __align__(16) float qs[4][kHeadDim];
+    extern __shared__ __align__(128) uint8_t pf_smem[];   // 2 stages x (K tile, V tile)
     pdl_wait();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long unit = (long)blockIdx.x * 4 + warp;
-    if (unit >= (long)rows * nq) return;
-    const int row = (int)(unit / nq), head = (int)(unit % nq);
-    const int seq = row / rows_per_seq;
-    const int pos = *d_len + row % rows_per_seq;
-    const int G = nq / nkv, j = head / G;
-    const int heads = nq + 2 * nkv;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int qt = gridDim.x - 1 - blockIdx.x;   // longest rows first
+    const int h = blockIdx.y, seq = blockIdx.z;
+    const int T = rows_per_seq, P0 = *d_len;
+    const int G = nq / nkv, j = h / G, heads = nq + 2 * nkv;
+    const int q0 = qt * kBM;
+    const int r0 = q0 + warp * 16 + g, r1 = r0 + 8;   // this thread's two query rows (token index inside the call)
+
+    // ---- Q fragments (pre-scaled so that exp2 can be used), as value + residual ----
     const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
+    uint32_t qh[8][4], ql[8][4];
     {
-        const float4 v = reinterpret_cast<const float4 *>(qkv + (size_t)row * heads * kHeadDim + (size_t)head * kHeadDim)[lane];
-        reinterpret_cast<float4 *>(qs[warp])[lane] = make_float4(v.x * qscale, v.y * qscale, v.z * qscale, v.w * qscale);
+        const float *qa = qkv + ((size_t)seq * T + min(r0, T - 1)) * heads * kHeadDim + (size_t)h * kHeadDim;
+        const float *qb = qkv + ((size_t)seq * T + min(r1, T - 1)) * heads * kHeadDim + (size_t)h * kHeadDim;
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const float2 a0 = *reinterpret_cast<const float2 *>(qa + 16 * s + 2 * t);
+            const float2 a2 = *reinterpret_cast<const float2 *>(qa + 16 * s + 2 * t + 8);
+            const float2 a1 = *reinterpret_cast<const float2 *>(qb + 16 * s + 2 * t);
+            const float2 a3 = *reinterpret_cast<const float2 *>(qb + 16 * s + 2 * t + 8);
+            split_pair(a0.x * qscale, a0.y * qscale, qh[s][0], ql[s][0]);
+            split_pair(a1.x * qscale, a1.y * qscale, qh[s][1], ql[s][1]);
+            split_pair(a2.x * qscale, a2.y * qscale, qh[s][2], ql[s][2]);
+            split_pair(a3.x * qscale, a3.y * qscale, qh[s][3], ql[s][3]);
+        }
     }
-    __syncwarp();
+
+    const int n_keys = min(P0 + q0 + kBM, P0 + T);       // cache positions the last row of this tile may see
+    const int n_tiles = (n_keys + kBN - 1) / kBN;
     const size_t head_off = ((size_t)seq * nkv + j) * (size_t)max_seq * kHeadDim;
-    const bf16 *kb = kcache + head_off, *vb = vcache + head_off;
-    float m = -INFINITY, l = 0.f;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int n_ctx = pos + 1;
-    for (int t0 = 0; t0 < n_ctx; t0 += 32) {
-        const int p = t0 + lane;
-        float s = -INFINITY;
-        if (p < n_ctx) {
-            const uint4 *kr = reinterpret_cast<const uint4 *>(kb + (size_t)p * kHeadDim);
-            float d = 0.f;
+    const bf16 *kbase = kcache + head_off, *vbase = vcache + head_off;
+    const uint32_t smem0 = smem_addr(pf_smem);
+
+    float o[16][4];
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const uint4 u = kr[c];
-                const float4 a = reinterpret_cast<const float4 *>(qs[warp])[2 * c];
-                const float4 b = reinterpret_cast<const float4 *>(qs[warp])[2 * c + 1];
-                d = fmaf(bf16_lo(u.x), a.x, d); d = fmaf(bf16_hi(u.x), a.y, d);
-                d = fmaf(bf16_lo(u.y), a.z, d); d = fmaf(bf16_hi(u.y), a.w, d);
-                d = fmaf(bf16_lo(u.z), b.x, d); d = fmaf(bf16_hi(u.z), b.y, d);
-                d = fmaf(bf16_lo(u.w), b.z, d); d = fmaf(bf16_hi(u.w), b.w, d);
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows r0, r1; l is a per-lane partial
+
+    load_tile(smem0, kbase, vbase, 0, n_keys - 1, tid);
+    cp_async_commit();
+
+    for (int kt = 0; kt < n_tiles; ++kt) {
+        const uint32_t st = smem0 + (uint32_t)(kt & 1) * 2u * kTileBytes;
+        if (kt + 1 < n_tiles) {
+            load_tile(smem0 + (uint32_t)((kt + 1) & 1) * 2u * kTileBytes, kbase, vbase, (kt + 1) * kBN, n_keys - 1, tid);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const int k0 = kt * kBN;
+        const int row_lo = P0 + q0 + warp * 16;           // absolute position of this warp's first query row
+        if (k0 <= row_lo + 15) {                          // warp-uniform: the tile holds something this warp may see
+            // ---- S = Q K^T over the 64 positions of the tile ----
+            float sacc[8][4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t kb[4];
+                    const int mi = lane >> 3;
+                    ldsm_x4(kb, st + tile_off(16 * np + (mi >> 1) * 8 + (lane & 7), 2 * s + (mi & 1)));
+                    mma16816(sacc[2 * np], qh[s], kb[0], kb[1]);
+                    mma16816(sacc[2 * np], ql[s], kb[0], kb[1]);
+                    mma16816(sacc[2 * np + 1], qh[s], kb[2], kb[3]);
+                    mma16816(sacc[2 * np + 1], ql[s], kb[2], kb[3]);
+                }
             }
-            s = d;
-        }
-        const float m_new = fmaxf(m, warp_max(s));
-        const float pr = exp2f(s - m_new);
-        const float alpha = exp2f(m - m_new);
-        l = l * alpha + warp_sum(pr);
-        m = m_new;
+            // ---- causal mask (diagonal tiles only), online softmax ----
+            if (k0 + kBN - 1 > row_lo) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i] *= alpha;
-        const int nv = min(32, n_ctx - t0);
-        for (int t = 0; t < nv; ++t) {
-            const float pt = __shfl_sync(0xffffffffu, pr, t);
-            const uint2 u = reinterpret_cast<const uint2 *>(vb + (size_t)(t0 + t) * kHeadDim)[lane];
-            acc[0] = fmaf(pt, bf16_lo(u.x), acc[0]);
-            acc[1] = fmaf(pt, bf16_hi(u.x), acc[1]);
-            acc[2] = fmaf(pt, bf16_lo(u.y), acc[2]);
-            acc[3] = fmaf(pt, bf16_hi(u.y), acc[3]);
+                for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int kabs = k0 + nt * 8 + 2 * t + e;
+                        if (kabs > P0 + r0) sacc[nt][e] = -INFINITY;
+                        if (kabs > P0 + r1) sacc[nt][2 + e] = -INFINITY;
+                    }
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite from the first tile on (key 0 is visible)
+            const float al0 = exp2f(m0 - mn0), al1 = exp2f(m1 - mn1);
+            m0 = mn0; m1 = mn1;
+            float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                sacc[nt][0] = exp2f(sacc[nt][0] - mn0); sacc[nt][1] = exp2f(sacc[nt][1] - mn0);
+                sacc[nt][2] = exp2f(sacc[nt][2] - mn1); sacc[nt][3] = exp2f(sacc[nt][3] - mn1);
+                sum0 += sacc[nt][0] + sacc[nt][1];
+                sum1 += sacc[nt][2] + sacc[nt][3];
+            }
+            l0 = l0 * al0 + sum0; l1 = l1 * al1 + sum1;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { o[i][0] *= al0; o[i][1] *= al0; o[i][2] *= al1; o[i][3] *= al1; }
+            // ---- O += P V ----
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                uint32_t ph[4], pl[4];
+                split_pair(sacc[2 * kk][0], sacc[2 * kk][1], ph[0], pl[0]);
+                split_pair(sacc[2 * kk][2], sacc[2 * kk][3], ph[1], pl[1]);
+                split_pair(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1], ph[2], pl[2]);
+                split_pair(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3], ph[3], pl[3]);
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    uint32_t vb[4];
+                    const int mi = lane >> 3;
+                    ldsm_x4_trans(vb, st + kTileBytes + tile_off(16 * kk + (mi & 1) * 8 + (lane & 7), 2 * dp + (mi >> 1)));
+                    mma16816(o[2 * dp], ph, vb[0], vb[1]);
+                    mma16816(o[2 * dp], pl, vb[0], vb[1]);
+                    mma16816(o[2 * dp + 1], ph, vb[2], vb[3]);
+                    mma16816(o[2 * dp + 1], pl, vb[2], vb[3]);
+                }
+            }
         }
+        __syncthreads();   // the other stage is refilled at the top of the next iteration
     }
-    const float inv = 1.f / l;
-    uint2 o;
-    o.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-    o.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-    const size_t oi = (size_t)row * nq * kHeadDim + (size_t)head * kHeadDim;
-    reinterpret_cast<uint2 *>(out + oi)[lane] = o;
-    if (out_lo) {  // rounding residual: out + out_lo carries 16 mantissa bits
-        uint2 r;
-        r.x = pack_bf16x2(acc[0] * inv - bf16_lo(o.x), acc[1] * inv - bf16_hi(o.x));
-        r.y = pack_bf16x2(acc[2] * inv - bf16_lo(o.y), acc[3] * inv - bf16_hi(o.y));
-        reinterpret_cast<uint2 *>(out_lo + oi)[lane] = r;
+
+    // ---- normalise and store as value + residual bf16 ----
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const float i0 = 1.f / l0, i1 = 1.f / l1;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int r = half ? r1 : r0;
+        if (r >= T) continue;
+        const float inv = half ? i1 : i0;
+        const size_t base = ((size_t)seq * T + r) * nq * kHeadDim + (size_t)h * kHeadDim + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            uint32_t hi, lo;
+            split_pair(o[nt][2 * half] * inv, o[nt][2 * half + 1] * inv, hi, lo);
+            *reinterpret_cast<uint32_t *>(out + base + nt * 8) = hi;
+            if (out_lo) *reinterpret_cast<uint32_t *>(out_lo + base + nt * 8) = lo;
+        }
     }
 }
 
@@ -90,9 +230,26 @@ attn_prefill_kernel(const float *__restrict__ qkv, int rows, int rows_per_seq, c
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
                                 const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
                                 const int32_t *d_len) {
-    const long units = (long)rows * nq;
-    return launch(lc, attn_prefill_kernel, dim3((unsigned)((units + 3) / 4)), dim3(128), qkv, rows, rows_per_seq,
-                  kcache, vcache, out, out_lo, nq, nkv, max_seq, d_len);
+    static bool attr_done = false;
+    const int smem = 4 * kTileBytes;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(attn_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const int batch = rows / rows_per_seq;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((rows_per_seq + kBM - 1) / kBM, nq, batch);
+    cfg.blockDim = dim3(kPfWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    if (lc.launches) ++*lc.launches;
+    return cudaLaunchKernelEx(&cfg, attn_prefill_kernel, qkv, rows_per_seq, kcache, vcache, out, out_lo, nq, nkv, max_seq, d_len);
 }
 
 }  // namespace nnc
