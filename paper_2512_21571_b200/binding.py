@@ -63,6 +63,8 @@ EXPORTS = {
                               C.c_int32, C.c_void_p]),
     "nnc_op_gemm_swiglu": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_void_p]),
+    "nnc_op_gemm_splitk": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                     C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "nnc_op_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "nnc_op_gemv": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_float, C.c_int32,
                               C.c_void_p]),
@@ -294,3 +296,17 @@ def op_attn_decode_static(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.T
                                       out.data_ptr(), batch, nq, nkv, max_seq, n_ctx, _stream_ptr()),
         "nnc_op_attn_decode_static")
     return out
+
+
+def op_gemm_splitk(X: torch.Tensor, W: torch.Tensor, scratch: torch.Tensor, out_f32: bool = True,
+                   accumulate_into: Optional[torch.Tensor] = None, X_lo: Optional[torch.Tensor] = None):
+    """nnc_op_gemm_splitk; `scratch` is a uint8 CUDA tensor whose first 16 KiB are zero."""
+    T, K = X.shape
+    N = W.shape[0]
+    Y = accumulate_into if accumulate_into is not None else \
+        torch.empty(T, N, dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
+    _ok(lib.nnc_op_gemm_splitk(_dev(X, torch.bfloat16), _dev(X_lo, torch.bfloat16) if X_lo is not None else None,
+                               _dev(W, torch.bfloat16), Y.data_ptr(), T, N, K, int(out_f32),
+                               int(accumulate_into is not None), scratch.data_ptr(), scratch.numel(), _stream_ptr()),
+        "nnc_op_gemm_splitk")
+    return Y

@@ -129,16 +129,20 @@ struct GemmParams {
     int T, N, K;      // tokens, weight rows, reduction
     int ldy;          // output row stride in elements
     int m_tiles, n_tiles;
+    int ksplit;          // K is cut into ksplit pieces per output tile (SWAP only); 1 = no split
+    float *part;         // ksplit > 1: fp32 partial tiles [tile][piece][BN / 32][128 rows][32]
+    uint32_t *tickets;   // ksplit > 1: one arrival counter per output tile, zero at rest
     int *status;
 };
 
 // Shared-memory stage: [weight tile][activation tile][activation residual tile (SPLIT)].
 // SWAP puts the weights on the M side (128 rows) and BN tokens on the N side; otherwise 128 tokens x BN weights.
-template <int BN, bool SWAP, bool SPLIT>
+template <int BN, bool SWAP, bool SPLIT, int KA>
 struct SmemLayout {
     static constexpr int kW = (SWAP ? kBM : BN) * kBK * 2;
     static constexpr int kX = (SWAP ? BN : kBM) * kBK * 2;
-    static constexpr int kStage = kW + kX * (SPLIT ? 2 : 1);
+    static constexpr int kAtom = kW + kX * (SPLIT ? 2 : 1);   // one 64-wide K slab of every operand
+    static constexpr int kStage = KA * kAtom;                 // KA slabs per pipeline stage
     static constexpr int kStagesFit = (192 * 1024) / kStage;
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr int kBytes = kStages * kStage + 1024 /*align slack*/ + 256 /*barriers*/;
@@ -150,11 +154,11 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + 
 // EPI: 0 fp32 store, 1 bf16 store, 2 fp32 accumulate (Y += D), 3 SwiGLU on interleaved gate/up weight rows -> bf16
 // SPLIT: the activations come as two bf16 matrices (value and rounding residual); both are multiplied with the
 // same weight tile into the same accumulator, which restores ~16 mantissa bits on the activation side.
-template <int BN, bool SWAP, int EPI, bool SPLIT>
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_x_lo, GemmParams p) {
-    using L = SmemLayout<BN, SWAP, SPLIT>;
+    using L = SmemLayout<BN, SWAP, SPLIT, KA>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = base + L::kStages * L::kStage;      // full[S], empty[S], tfull[2], tempty[2], 8 B each
@@ -164,6 +168,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * L::kStages + 2 + a); };
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ bool split_last;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
@@ -186,8 +191,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    const int kb_count = p.K / kBK;
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int kb_count = p.K / (kBK * KA);   // pipeline stages along K
+    const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;   // work units: (output tile, K piece)
+    // unit u -> output tile u / ksplit (m fastest), K blocks [kb_lo, kb_hi)
+#define NNC_UNIT_DECODE(u)                                                        \
+    const int tile_id = (u) / p.ksplit, ks_id = (u) % p.ksplit;                   \
+    const int mt = tile_id % p.m_tiles, nt = tile_id / p.m_tiles;                 \
+    const int kb_lo = ks_id * kb_count / p.ksplit, kb_hi = (ks_id + 1) * kb_count / p.ksplit;
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
@@ -195,16 +205,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+                NNC_UNIT_DECODE(tile)
                 const int w_row = SWAP ? mt * kBM : nt * BN;
                 const int x_row = SWAP ? nt * BN : mt * kBM;
-                for (int kb = 0; kb < kb_count; ++kb) {
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     mbar_expect_tx(full_bar(stage), L::kStage);
                     const uint32_t sw = base + stage * L::kStage;
-                    tma_load_2d(sw, &map_w, full_bar(stage), kb * kBK, w_row);
-                    tma_load_2d(sw + L::kW, &map_x, full_bar(stage), kb * kBK, x_row);
-                    if (SPLIT) tma_load_2d(sw + L::kW + L::kX, &map_x_lo, full_bar(stage), kb * kBK, x_row);
+#pragma unroll
+                    for (int a = 0; a < KA; ++a) {   // KA consecutive slabs: KA * 128 contiguous bytes of every weight row
+                        const uint32_t sa = sw + a * L::kAtom;
+                        const int kx = (kb * KA + a) * kBK;
+                        tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
+                        tma_load_2d(sa + L::kW, &map_x, full_bar(stage), kx, x_row);
+                        if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage), kx, x_row);
+                    }
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -219,21 +234,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < kb_count; ++kb) {
+                NNC_UNIT_DECODE(tile)
+                (void)mt; (void)nt;
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sw = base + stage * L::kStage;
-                    const uint64_t dw = make_smem_desc(sw), dx = make_smem_desc(sw + L::kW),
-                                   dxl = make_smem_desc(sw + L::kW + L::kX);
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k) {
-                        const uint64_t off = (uint64_t)(k * 2);  // 32 bytes, in 16-byte units
-                        if (SWAP) {
-                            umma_bf16(d_tmem, dw + off, dx + off, idesc, (kb | k) != 0);
-                            if (SPLIT) umma_bf16(d_tmem, dw + off, dxl + off, idesc, 1u);
-                        } else {
-                            umma_bf16(d_tmem, dx + off, dw + off, idesc, (kb | k) != 0);
-                            if (SPLIT) umma_bf16(d_tmem, dxl + off, dw + off, idesc, 1u);
+                    for (int a = 0; a < KA; ++a) {
+                        const uint32_t sa = sw + a * L::kAtom;
+                        const uint64_t dw = make_smem_desc(sa), dx = make_smem_desc(sa + L::kW),
+                                       dxl = make_smem_desc(sa + L::kW + L::kX);
+#pragma unroll
+                        for (int k = 0; k < kBK / 16; ++k) {
+                            const uint64_t off = (uint64_t)(k * 2);  // 32 bytes, in 16-byte units
+                            const uint32_t accum = (kb != kb_lo) || (a != 0) || (k != 0);
+                            if (SWAP) {
+                                umma_bf16(d_tmem, dw + off, dx + off, idesc, accum);
+                                if (SPLIT) umma_bf16(d_tmem, dw + off, dxl + off, idesc, 1u);
+                            } else {
+                                umma_bf16(d_tmem, dx + off, dw + off, idesc, accum);
+                                if (SPLIT) umma_bf16(d_tmem, dxl + off, dw + off, idesc, 1u);
+                            }
                         }
                     }
                     umma_commit(empty_bar(stage));
@@ -248,11 +270,107 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int quarter = warp & 3;  // TMEM lane quarter this warp may read
         int acc = 0;
         uint32_t acc_phase = 0;
+        // SWAP stores: row m = weight row, columns = tokens n0 .. n0 + 31; a warp stores 32 consecutive weight rows per token
+        auto store_swap = [&](const uint32_t (&r)[32], int m, int n0) {
+            if (EPI == 3) {
+                // gate in even lanes, up in odd lanes
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float mine = __uint_as_float(r[i]);
+                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                    const int t = n0 + i;
+                    if (!(lane & 1) && m + 1 < p.N && t < p.T) {
+                        const float a = silu_mul(mine, other);
+                        const bf16 hi = __float2bfloat16_rn(a);
+                        const size_t yo = (size_t)t * p.ldy + (m >> 1);
+                        reinterpret_cast<bf16 *>(p.Y)[yo] = hi;
+                        if (p.Y_lo) reinterpret_cast<bf16 *>(p.Y_lo)[yo] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int t = n0 + i;
+                    if (m < p.N && t < p.T) {
+                        const float v = __uint_as_float(r[i]);
+                        if (EPI == 1) reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + m] = __float2bfloat16_rn(v);
+                        else if (EPI == 2) reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] += v;
+                        else reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] = v;
+                    }
+                }
+            }
+        };
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
-            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
+            NNC_UNIT_DECODE(tile)
+            (void)kb_lo; (void)kb_hi;
+            const bool got = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4);
+            if (!got && !(SWAP && p.ksplit > 1)) break;
             tc_fence_after();
             const int m = mt * kBM + quarter * 32 + lane;  // D row held by this thread
+            if (SWAP && p.ksplit > 1) {
+                // ---- split K: park this piece's fp32 tile, take a ticket; the piece that arrives last adds the
+                //      pieces in piece order and runs the epilogue (nobody waits) ----
+                const int row = quarter * 32 + lane;
+                float *slot = p.part + ((size_t)tile_id * p.ksplit + ks_id) * (size_t)(BN * kBM);
+                if (got) {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                        uint4 *dst = reinterpret_cast<uint4 *>(slot + ((size_t)(c0 >> 5) * kBM + row) * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));
+                }
+                __threadfence();
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (*abort_flag) break;
+                if (warp == 2 && lane == 0) {
+                    const unsigned tk = atomicAdd(&p.tickets[tile_id], 1u);
+                    split_last = (tk == (unsigned)p.ksplit - 1);
+                    if (split_last) p.tickets[tile_id] = 0u;
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (split_last) {
+                    __threadfence();
+                    const float *base = p.part + (size_t)tile_id * p.ksplit * (size_t)(BN * kBM);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN; c0 += 32) {
+                        float sum[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) sum[i] = 0.f;
+                        // pieces are added in piece order; two pieces' loads are in flight at a time
+                        for (int ks = 0; ks < p.ksplit; ks += 2) {
+                            const float4 *s0 = reinterpret_cast<const float4 *>(base + (size_t)ks * (BN * kBM) + ((size_t)(c0 >> 5) * kBM + row) * 32);
+                            const bool two = ks + 1 < p.ksplit;
+                            const float4 *s1 = two ? s0 + (BN * kBM) / 4 : s0;
+                            float4 v0[8], v1[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) { v0[i] = __ldcg(s0 + i); v1[i] = __ldcg(s1 + i); }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                sum[4 * i] += v0[i].x; sum[4 * i + 1] += v0[i].y; sum[4 * i + 2] += v0[i].z; sum[4 * i + 3] += v0[i].w;
+                            }
+                            if (two) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    sum[4 * i] += v1[i].x; sum[4 * i + 1] += v1[i].y; sum[4 * i + 2] += v1[i].z; sum[4 * i + 3] += v1[i].w;
+                                }
+                            }
+                        }
+                        uint32_t r[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i]);
+                        store_swap(r, m, nt * BN + c0);
+                    }
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");   // split_last is rewritten by the next unit
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                continue;
+            }
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
@@ -325,34 +443,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         }
                     }
                 } else {
-                    // row m = weight row, columns = tokens: a warp stores 32 consecutive weight rows per token
-                    if (EPI == 3) {
-                        // gate in even lanes, up in odd lanes
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float mine = __uint_as_float(r[i]);
-                            const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                            const int t = n0 + i;
-                            if (!(lane & 1) && m + 1 < p.N && t < p.T) {
-                                const float a = silu_mul(mine, other);
-                                const bf16 hi = __float2bfloat16_rn(a);
-                                const size_t yo = (size_t)t * p.ldy + (m >> 1);
-                                reinterpret_cast<bf16 *>(p.Y)[yo] = hi;
-                                if (p.Y_lo) reinterpret_cast<bf16 *>(p.Y_lo)[yo] = __float2bfloat16_rn(a - __bfloat162float(hi));
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int t = n0 + i;
-                            if (m < p.N && t < p.T) {
-                                const float v = __uint_as_float(r[i]);
-                                if (EPI == 1) reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + m] = __float2bfloat16_rn(v);
-                                else if (EPI == 2) reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] += v;
-                                else reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] = v;
-                            }
-                        }
-                    }
+                    store_swap(r, m, n0);
                 }
             }
             tc_fence_before();
@@ -409,11 +500,11 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows) 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool SWAP, int EPI, bool SPLIT>
-cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
-                      int K, int ldy, int *status) {
-    using L = SmemLayout<BN, SWAP, SPLIT>;
-    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT>;
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA>
+cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
+                      int K, int ldy, int *status, const GemmScratch *scratch) {
+    using L = SmemLayout<BN, SWAP, SPLIT, KA>;
+    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes);
@@ -433,30 +524,59 @@ cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, cons
         p.m_tiles = (N + kBM - 1) / kBM;
         p.n_tiles = (T + BN - 1) / BN;
     }
-    int grid = p.m_tiles * p.n_tiles;
+    // Few tokens: the product is bound by streaming the weights, and N / 128 output tiles are too few to keep every
+    // SM's loads in flight.  Cut K into pieces so that (tiles x pieces) fills the SMs in whole rounds.
+    p.ksplit = 1; p.part = nullptr; p.tickets = nullptr;
+    if (SWAP && scratch && scratch->part && scratch->tickets) {
+        const int tiles = p.m_tiles * p.n_tiles, kb_count = K / (kBK * KA);
+        const size_t slot_bytes = (size_t)BN * kBM * 4;
+        double best = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
+        for (int ks = 2; ks <= 16 && best < 0.95; ++ks) {
+            if (kb_count / ks < 2) break;
+            if ((size_t)tiles * ks * slot_bytes > scratch->part_bytes || tiles > scratch->n_tickets) break;
+            const int units = tiles * ks;
+            const double eff = (double)units / (((units + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
+            if (eff > best + 0.02) { best = eff; p.ksplit = ks; }
+        }
+        if (p.ksplit > 1) { p.part = scratch->part; p.tickets = scratch->tickets; }
+    }
+    int grid = p.m_tiles * p.n_tiles * p.ksplit;
     if (grid > lc.sm_count) grid = lc.sm_count;
     if (lc.launches) ++*lc.launches;
     kern<<<grid, kGemmThreads, L::kBytes, lc.stream>>>(map_w, map_x, map_x_lo, p);
     return cudaGetLastError();
 }
 
+// Few tokens (weights on the M side): a stage carries 4 (<= 32 tokens) or 2 (<= 64) consecutive K slabs, so that
+// every weight row is fetched in 512 / 256 contiguous bytes instead of 128 -- the product is HBM-bound there and
+// DRAM efficiency follows the contiguous run length.
+template <int BN, bool SWAP, int EPI, bool SPLIT>
+cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
+                      int K, int ldy, int *status, const GemmScratch *scratch) {
+    if (SWAP && BN == 32 && K % (4 * kBK) == 0)
+        return launch_tc_ka<BN, SWAP, EPI, SPLIT, (SWAP && BN == 32) ? 4 : 1>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, scratch);
+    if (SWAP && BN == 64 && K % (2 * kBK) == 0)
+        return launch_tc_ka<BN, SWAP, EPI, SPLIT, (SWAP && BN == 64) ? 2 : 1>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, scratch);
+    return launch_tc_ka<BN, SWAP, EPI, SPLIT, 1>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, scratch);
+}
+
 template <int EPI, bool SPLIT>
 cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
-                     int K, int ldy, int *status) {
-    if (T <= 32) return launch_tc<32, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-    if (T <= 64) return launch_tc<64, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-    if (T <= 128) return launch_tc<128, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-    return launch_tc<256, false, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+                     int K, int ldy, int *status, const GemmScratch *sc) {
+    if (T <= 32) return launch_tc<32, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+    if (T <= 64) return launch_tc<64, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+    if (T <= 128) return launch_tc<128, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+    return launch_tc<256, false, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
 }
 
 template <bool SPLIT>
 cudaError_t dispatch_epi(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                         int N, int K, int ldy, int epi, int *status) {
+                         int N, int K, int ldy, int epi, int *status, const GemmScratch *sc) {
     switch (epi) {
-        case kEpiStoreF32: return dispatch<0, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-        case kEpiStoreBf16: return dispatch<1, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-        case kEpiAccumF32: return dispatch<2, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
-        case kEpiSwigluBf16: return dispatch<3, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status);
+        case kEpiStoreF32: return dispatch<0, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+        case kEpiStoreBf16: return dispatch<1, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+        case kEpiAccumF32: return dispatch<2, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+        case kEpiSwigluBf16: return dispatch<3, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
     }
     return cudaErrorInvalidValue;
 }
@@ -467,15 +587,15 @@ bool gemm_tc_available() { return get_encode() != nullptr; }
 
 // Y[T][*] (row stride ldy) = epilogue((X + X_lo)[T][K] * W[N][K]^T).  Operands 16-byte aligned, K % 64 == 0.
 cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                        int N, int K, int ldy, int epi, int *status) {
+                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch) {
     if (T <= 0 || N <= 0 || K <= 0 || K % kBK != 0 || N % 8 != 0) return cudaErrorInvalidValue;
     if (((uintptr_t)X | (uintptr_t)X_lo | (uintptr_t)W | (uintptr_t)Y | (uintptr_t)Y_lo) & 15) return cudaErrorInvalidValue;
     // the epilogue stores 16-byte vectors per output row: the row pitch must keep them aligned
     const bool out_bf16 = epi == kEpiStoreBf16 || epi == kEpiSwigluBf16;
     if (ldy % (out_bf16 ? 8 : 4) != 0) return cudaErrorInvalidValue;
     if (epi == kEpiSwigluBf16 && N % 2 != 0) return cudaErrorInvalidValue;
-    return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status)
-                : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status);
+    return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch)
+                : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch);
 }
 
 }  // namespace nnc

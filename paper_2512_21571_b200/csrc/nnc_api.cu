@@ -32,7 +32,7 @@ struct Plan {
     // offsets
     std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
-    size_t gemv_ctr, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
+    size_t gemv_ctr, gemm_part, gemm_tickets, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
     size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
     size_t take(size_t bytes) {
         const size_t o = total;
@@ -76,6 +76,8 @@ void make_plan(const nnc_config &c, Plan &p) {
     p.vcache = p.take(kv);
     p.rope = p.take((size_t)c.max_seq * 128 * 4);
     p.gemv_ctr = p.take(((size_t)c.n_layers * 4 + 2) * 16);
+    p.gemm_part = p.take(c.max_tokens > 0 ? kGemmPartBytes : 0);
+    p.gemm_tickets = p.take((size_t)kGemmTickets * 4);
     p.x = p.take(H * 4);
     p.qkv = p.take(qkvd * 4);
     p.attn_out = p.take(qd * 4);
@@ -113,6 +115,7 @@ struct nnc_model {
     bf16 *embed, *lm_head, *g_final, *kcache, *vcache;
     float *rope, *x, *qkv, *attn_out, *act, *part;
     uint32_t *tickets;
+    GemmScratch gemm_scratch;  // split-K partial tiles and tickets of the token-batch GEMMs
     uint32_t *gemv_ctr;  // 4 words per GEMV call site (4 per layer + lm_head): dynamic work counters, zero at rest
     ArgmaxScratch am;
     int32_t *d_len, *d_status, *d_tokens, *d_argmax;
@@ -204,7 +207,7 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
         bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
         bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
         NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_in, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
-        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wqkv, m->qkvt, nullptr, R, qkvd, H, qkvd, kEpiStoreF32, m->d_status));
+        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wqkv, m->qkvt, nullptr, R, qkvd, H, qkvd, kEpiStoreF32, m->d_status, &m->gemm_scratch));
         if (T == 1) {
             const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
             NNC_CUDA(m, launch_attn_decode(lc, m->qkvt, qkvd, kc, vc, nullptr, m->ob, m->ob_lo, qd, m->part, m->tickets, m->d_len, 1,
@@ -214,23 +217,23 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
                                                    c.n_kv_heads, c.max_seq, m->d_len, nullptr));
             NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, c.n_q_heads, c.n_kv_heads, c.max_seq, m->d_len));
         }
-        NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status));
+        NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
         NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
-        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wgu, m->ab, m->ab_lo, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status));
-        NNC_CUDA(m, launch_gemm(lc, m->ab, m->ab_lo, w.wd, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status));
+        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wgu, m->ab, m->ab_lo, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status, &m->gemm_scratch));
+        NNC_CUDA(m, launch_gemm(lc, m->ab, m->ab_lo, w.wd, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
         if (m->taps) NNC_CUDA(m, launch_copy_f32(lc, m->xt, m->taps + (size_t)(l + 1) * R * H, (size_t)R * H));
     }
     if (logits) {
         if (all_positions || T == 1) {
             NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
-            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, R, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, R, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status, &m->gemm_scratch));
         } else if (batch == 1) {
             // last position only: the streaming GEMV keeps the activation in fp32
             NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->xt + (size_t)(T - 1) * H, logits, c.vocab, H, m->g_final, c.rms_eps,
                                     kGemvLogits, nullptr));
         } else {
             NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, m->hb_lo, batch, H, c.rms_eps, T - 1, T));
-            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, batch, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, batch, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status, &m->gemm_scratch));
         }
     }
     NNC_CUDA(m, launch_add_len(lc, m->d_len, T));
@@ -303,6 +306,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         m->x = (float *)at(p.x); m->qkv = (float *)at(p.qkv); m->attn_out = (float *)at(p.attn_out);
         m->act = (float *)at(p.act); m->part = (float *)at(p.part); m->tickets = (uint32_t *)at(p.tickets);
         m->gemv_ctr = (uint32_t *)at(p.gemv_ctr);
+        m->gemm_scratch = GemmScratch{(float *)at(p.gemm_part), kGemmPartBytes, (uint32_t *)at(p.gemm_tickets), kGemmTickets};
         m->am = ArgmaxScratch{(float *)at(p.am_val), (int32_t *)at(p.am_idx), (uint32_t *)at(p.am_ticket), nullptr};
         m->d_len = (int32_t *)at(p.d_len); m->d_status = (int32_t *)at(p.d_status);
         m->d_tokens = (int32_t *)at(p.d_tokens); m->d_argmax = (int32_t *)at(p.d_argmax);
@@ -357,6 +361,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         }
         NNC_CUDA(m, cudaMemsetAsync(m->tickets, 0, (size_t)c.max_batch * c.n_kv_heads * 4, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->am.ticket, 0, 4, m->stream));
+        NNC_CUDA(m, cudaMemsetAsync(m->gemm_scratch.tickets, 0, (size_t)kGemmTickets * 4, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->gemv_ctr, 0, ((size_t)c.n_layers * 4 + 2) * 16, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->d_len, 0, 4, m->stream));
         NNC_CUDA(m, cudaMemsetAsync(m->d_status, 0, 4, m->stream));
@@ -649,6 +654,22 @@ int nnc_op_gemm_swiglu(const void *X, const void *X_lo, const void *W, void *Y, 
     int *status = nullptr;
     if (cudaGetSymbolAddress((void **)&status, g_op_status) != cudaSuccess) return NNC_ERR_CUDA;
     cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)X_lo, (const bf16 *)W, Y, Y_lo, T, n_out, n_in, n_out / 2, kEpiSwigluBf16, status);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
+int nnc_op_gemm_splitk(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                       int32_t out_f32, int32_t accumulate, void *scratch, size_t scratch_bytes, void *cuda_stream) {
+    if (!X || !W || !Y || !scratch || ((uintptr_t)scratch & 255)) return NNC_ERR_INVALID_ARG;
+    if (accumulate && !out_f32) return NNC_ERR_INVALID_ARG;
+    const size_t ticket_bytes = (size_t)kGemmTickets * 4;
+    if (scratch_bytes < ticket_bytes + (1u << 20)) return NNC_ERR_WORKSPACE;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    const GemmScratch sc{(float *)((char *)scratch + ticket_bytes), scratch_bytes - ticket_bytes, (uint32_t *)scratch, kGemmTickets};
+    const int epi = out_f32 ? (accumulate ? kEpiAccumF32 : kEpiStoreF32) : kEpiStoreBf16;
+    cudaError_t e = launch_gemm(lc, (const bf16 *)X, (const bf16 *)X_lo, (const bf16 *)W, Y, nullptr, T, n_out, n_in, n_out, epi,
+                                lc.status, &sc);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }

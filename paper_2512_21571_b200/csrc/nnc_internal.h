@@ -92,8 +92,18 @@ enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwiglu
 bool gemm_tc_available();
 // X_lo (nullable): bf16 rounding residual of the activations; the product is then (X + X_lo) W^T.
 // Y_lo (nullable, SwiGLU epilogue only): receives the rounding residual of the bf16 output.
+// scratch (nullable): lets products with at most 128 tokens split K across CTAs (fp32 partial tiles + one ticket
+// word per output tile, zero at rest); without it every output tile is computed by one CTA.
+struct GemmScratch {
+    float *part;
+    size_t part_bytes;
+    uint32_t *tickets;
+    int n_tickets;
+};
+constexpr size_t kGemmPartBytes = 48u << 20;
+constexpr int kGemmTickets = 4096;
 cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                        int N, int K, int ldy, int epi, int *status);
+                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch = nullptr);
 
 // ---- repack (repack.cu) -------------------------------------------------------------------------------
 // dst rows [row0, row0 + rows) <- src rows [0, rows), row length K (plain row copy into a taller matrix)

@@ -143,3 +143,29 @@ def test_gemm_split_activations_recover_fp32_inputs(nnc, oracle_mod, T, N, K):
     refa = ref[:, 0::2] / (1 + torch.exp(-ref[:, 0::2])) * ref[:, 1::2]
     assert (A.double() + A_lo.double() - refa).abs().max().item() < 1e-4
     assert nnc.op_status() == 0
+
+
+@pytest.mark.parametrize("T,N,K", [(32, 4096, 4096), (7, 384, 640), (128, 1024, 2048), (33, 1000, 1024), (32, 4096, 12288)])
+def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
+    """Few tokens: K is cut into pieces across CTAs and the fp32 partial tiles are added in piece order.  Same
+    result as the oracle's matmul, bit-identical from run to run, scratch counters left at zero."""
+    X = synth.normal(8, 1, (T, K), 1.0, torch.float32, "cuda")
+    W = _w(8, 2, (N, K))
+    hi, lo = nnc.split_bf16(X)
+    scratch = torch.zeros(16384 + (32 << 20), dtype=torch.uint8, device="cuda")
+    Y = nnc.op_gemm_splitk(hi, W, scratch, X_lo=lo)
+    Y2 = nnc.op_gemm_splitk(hi, W, scratch, X_lo=lo)
+    torch.cuda.synchronize()
+    assert nnc.op_status() == 0
+    assert torch.equal(Y, Y2)
+    assert int(scratch[:16384].max()) == 0
+    rows = sorted(set([0, T - 1, T // 2]))
+    want = oracle_mod.matmul(W.cpu(), X[rows].cpu())
+    assert torch.allclose(Y[rows].cpu(), want, rtol=1e-4, atol=3e-5 * math.sqrt(K))
+    ref = X.double() @ W.double().T
+    assert (Y.double() - ref).abs().max().item() < 2e-5 * math.sqrt(K)
+    acc = synth.normal(8, 3, (T, N), 1.0, torch.float32, "cuda")
+    Y3 = nnc.op_gemm_splitk(hi, W, scratch, X_lo=lo, accumulate_into=acc.clone())
+    assert (Y3.double() - (acc.double() + ref)).abs().max().item() < 1e-4 * math.sqrt(K)
+    Yb = nnc.op_gemm_splitk(hi, W, scratch, out_f32=False)
+    assert torch.allclose(Yb.float(), ref.float(), rtol=2e-2, atol=2e-2)
