@@ -145,12 +145,20 @@ def barrier(world):
 
 
 def max_over_ranks(ms: float, world: int) -> float:
+    """Device time of the slowest rank (every rank returns the same number)."""
     if world == 1:
         return ms
     import torch.distributed as dist
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def whole_job_throughput(ms_local: float, steps: int, units_per_step: int, world: int):
+    """(ms of the slowest rank, units/s of all replicas together): every rank did `steps * units_per_step` units."""
+    ms = max_over_ranks(ms_local, world)
+    return ms, world * steps * units_per_step / (ms * 1e-3)
 
 
 def build_model(wl, max_tokens=None):
@@ -496,12 +504,10 @@ def main():
 
     if wl["kind"] == "decode":
         ms, launches, clocks = time_decode(m, shape, wl, steps, warmup, world)
-        ms = max_over_ranks(ms, world)
         units_per_step = wl["batch"]
-        value = world * steps * units_per_step / (ms * 1e-3)
+        ms, value = whole_job_throughput(ms, steps, units_per_step, world)
         ms_e, h2d, d2h = time_decode_e2e(m, shape, wl, steps, warmup, world)
-        ms_e = max_over_ranks(ms_e, world)
-        e2e_value = world * steps * units_per_step / (ms_e * 1e-3)
+        ms_e, e2e_value = whole_job_throughput(ms_e, steps, units_per_step, world)
         ctx_mid = wl["ctx"] + min(steps, wl["pass_steps"]) / 2.0
         nbytes = decode_bytes_per_step(shape, wl["batch"], ctx_mid)
         ach = nbytes / (ms / steps * 1e-3) / 1e9
@@ -510,12 +516,10 @@ def main():
                      "frac_of_nominal_8000": round(ach / 8000.0, 4)}
     else:
         ms, launches, clocks, h2d, d2h = time_prefill(m, shape, wl, steps, warmup, world)
-        ms = max_over_ranks(ms, world)
         units_per_step = wl["batch"] * wl["tokens"]
-        value = world * steps * units_per_step / (ms * 1e-3)
+        ms, value = whole_job_throughput(ms, steps, units_per_step, world)
         ms_e, _, _, h2d, d2h = time_prefill(m, shape, wl, steps, 1, world, host=True)
-        ms_e = max_over_ranks(ms_e, world)
-        e2e_value = world * steps * units_per_step / (ms_e * 1e-3)
+        ms_e, e2e_value = whole_job_throughput(ms_e, steps, units_per_step, world)
         proj, attn, head = prefill_flops(shape, wl["batch"], wl["tokens"])
         ach = (proj + attn + head) / (ms / steps * 1e-3) / 1e12
         step_roof = {"bound": "tensor", "flops_per_step": proj + attn + head, "projection_flops": proj,
