@@ -15,348 +15,39 @@
 //     partials in split order (a ticket counter; nobody waits), so the result does not depend on arrival order.
 //   - before waiting on the preceding kernel, the CTA asks for its K/V range to be brought into L2
 //     (cp.async.bulk.prefetch): the cache rows of earlier positions do not depend on that kernel.
-#include "common.cuh"
-#include "nnc_internal.h"
+#include "attn_decode_body.cuh"
 
 namespace nnc {
 
 namespace {
 
-constexpr int kPartStride = kHeadDim + 4;  // o~[128], m, l, 2 pad words (rows stay 16-byte aligned)
-constexpr int kWarps = 4;
-
-__device__ __forceinline__ uint4 ldg_cg(const void *p) {
-    uint4 v;
-    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-    // rows 8..15 of the 16-row operand are padding: a1 = a3 = 0
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
-
-// value + residual bf16 pairs of two floats: hi holds bf16(x), lo holds bf16(x - hi)
-__device__ __forceinline__ void split2(float x, float y, uint32_t &hi, uint32_t &lo) {
-    hi = pack_bf16x2(x, y);
-    lo = pack_bf16x2(x - bf16_lo(hi), y - bf16_hi(hi));
-}
-
-struct AttnParams {
-    const float *q;          // [batch][q_row_stride]: query heads first; FUSED: then key heads, then value heads (raw)
-    int q_row_stride;
-    bf16 *kcache, *vcache;   // this layer: [batch][nkv][max_seq][128]
-    float *out_f32;          // [batch][out_row_stride] or null
-    bf16 *out_bf16, *out_bf16_lo;
-    int out_row_stride;
-    float *part;
-    uint32_t *tickets;
-    const int32_t *d_len;    // cached positions before this call (null = 0)
-    int len_add;             // positions attended = *d_len + len_add
-    int nkv, max_seq, n_splits;
-    const bf16 *g_q, *g_k;   // FUSED: per-head RMSNorm gains
-    const float *rope;       // FUSED: [max_seq][64][2]
-    float eps;
-};
-
-// RMSNorm over the 128 elements of one head + rotation by the table row; lane l owns elements 2l, 2l+1 and their
-// rotation partners 2l+64, 2l+65 (half-split pairing).
-__device__ __forceinline__ void norm_rope(float2 &a, float2 &b, const bf16 *gain, const float *rope_row, float eps, int lane) {
-    const float ss = warp_sum(a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y);
-    const float inv = rsqrtf(ss * (1.f / kHeadDim) + eps);
-    const uint32_t ga = reinterpret_cast<const uint32_t *>(gain)[lane];
-    const uint32_t gb = reinterpret_cast<const uint32_t *>(gain + 64)[lane];
-    a.x *= inv * bf16_lo(ga); a.y *= inv * bf16_hi(ga);
-    b.x *= inv * bf16_lo(gb); b.y *= inv * bf16_hi(gb);
-    const float4 cs = reinterpret_cast<const float4 *>(rope_row)[lane];  // c0 s0 c1 s1
-    const float2 ra = make_float2(a.x * cs.x - b.x * cs.y, a.y * cs.z - b.y * cs.w);
-    const float2 rb = make_float2(b.x * cs.x + a.x * cs.y, b.y * cs.z + a.y * cs.w);
-    a = ra; b = rb;
-}
-
 template <int G, bool FUSED>
-__global__ void __launch_bounds__(kWarps * 32) attn_decode_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(const AttnParams p) {
     NNC_TRACE_SCOPE(30);
-    __shared__ __align__(16) float qs[G][kHeadDim];              // processed queries, pre-scaled for exp2
-    __shared__ float comb[kWarps][G][kPartStride];               // per-warp (o~, m, l)
-    __shared__ bool is_last;
-
+    __shared__ AttnSmem<G> sm;
     const int split = blockIdx.x, j = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g8 = lane >> 2, t4 = lane & 3;   // fragment coordinates: row / column group, and position inside it
-    const int nq = p.nkv * G;
-    const size_t head_off = ((size_t)b * p.nkv + j) * (size_t)p.max_seq * kHeadDim;
-    bf16 *kbase = p.kcache + head_off;
-    bf16 *vbase = p.vcache + head_off;
+    const int tid = threadIdx.x;
 
     pdl_launch_dependents();
     // ---- before the dependency: ask for this CTA's K/V range in L2 (rows of earlier positions are stable) ----
     {
+        const size_t head_off = ((size_t)b * p.nkv + j) * (size_t)p.max_seq * kHeadDim;
         const int n_guess = (p.d_len ? *p.d_len : 0) + p.len_add;   // only a hint here; read again after the wait
         int chunk = (n_guess + p.n_splits - 1) / p.n_splits;
         chunk = (chunk + 15) & ~15;
         if (chunk < 16) chunk = 16;
         const int c0 = split * chunk, c1 = min(c0 + chunk, min(n_guess, p.max_seq));
         if (tid < 2 && c1 > c0) {
-            const bf16 *src = (tid ? vbase : kbase) + (size_t)c0 * kHeadDim;
+            const bf16 *src = (tid ? p.vcache : p.kcache) + head_off + (size_t)c0 * kHeadDim;
             const uint32_t bytes = (uint32_t)(c1 - c0) * kHeadDim * 2u;
             asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
         }
     }
     pdl_wait();
     NNC_TRACE_MARK();
-
-    const int n_ctx = (p.d_len ? *p.d_len : 0) + p.len_add;
-    int chunk = (n_ctx + p.n_splits - 1) / p.n_splits;
-    chunk = (chunk + 15) & ~15;
-    if (chunk < 16) chunk = 16;
-    const int c0 = split * chunk;
-    const int c1 = min(c0 + chunk, n_ctx);
-    const int n_active = (n_ctx + chunk - 1) / chunk;
-    if (c0 >= n_ctx) return;  // whole CTA; takes no ticket (n_active counts only non-empty ranges)
-
-    // ---- K/V fragment loads of one block of 16 positions: K rows p0 + 8h + g8 (h = 0, 1), V rows
-    //      p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9}; rows past the range are clamped here and masked later ----
-    uint4 kf[2][4], vf[4][2];
-    auto load_block = [&](int p0) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int pos = min(p0 + 8 * h + g8, c1 - 1);
-            const bf16 *kr = kbase + (size_t)pos * kHeadDim + 8 * t4;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) kf[h][c] = ldg_cg(kr + 32 * c);
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int pos = min(p0 + 2 * t4 + (r & 1) + 8 * (r >> 1), c1 - 1);
-            const bf16 *vr = vbase + (size_t)pos * kHeadDim + 8 * g8;
-            vf[r][0] = ldg_cg(vr);
-            vf[r][1] = ldg_cg(vr + 64);
-        }
-    };
-    const int n_blocks = (c1 - c0 + 15) >> 4;
-    // the warp's first block is requested now and lands while the queries are prepared -- unless it holds the row
-    // that is appended below
-    const bool early = warp < n_blocks && !(FUSED && c0 + warp * 16 + 16 >= n_ctx);
-    if (early) load_block(c0 + warp * 16);
-
-    // ---- queries (and, fused, the new token's K/V row) ----
-    const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);   // scores in log2 units
-    const float *qrow = p.q + (size_t)b * p.q_row_stride;
-    for (int g = warp; g < G; g += kWarps) {
-        const float *src = qrow + (size_t)(j * G + g) * kHeadDim;
-        float2 a = reinterpret_cast<const float2 *>(src)[lane];
-        float2 c = reinterpret_cast<const float2 *>(src + 64)[lane];
-        if (FUSED) norm_rope(a, c, p.g_q, p.rope + (size_t)(n_ctx - 1) * kHeadDim, p.eps, lane);
-        reinterpret_cast<float2 *>(&qs[g][0])[lane] = make_float2(a.x * qscale, a.y * qscale);
-        reinterpret_cast<float2 *>(&qs[g][64])[lane] = make_float2(c.x * qscale, c.y * qscale);
-    }
-    if (FUSED && split == n_active - 1) {
-        // this CTA's range ends with the new position: normalise + rotate its key, round both rows to bf16, append
-        const int pos = n_ctx - 1;
-        if (warp == (G % kWarps)) {
-            const float *src = qrow + (size_t)(nq + j) * kHeadDim;
-            float2 a = reinterpret_cast<const float2 *>(src)[lane];
-            float2 c = reinterpret_cast<const float2 *>(src + 64)[lane];
-            norm_rope(a, c, p.g_k, p.rope + (size_t)pos * kHeadDim, p.eps, lane);
-            bf16 *dst = kbase + (size_t)pos * kHeadDim;
-            reinterpret_cast<uint32_t *>(dst)[lane] = pack_bf16x2(a.x, a.y);
-            reinterpret_cast<uint32_t *>(dst + 64)[lane] = pack_bf16x2(c.x, c.y);
-        }
-        if (warp == ((G + 1) % kWarps)) {
-            const float *src = qrow + (size_t)(nq + p.nkv + j) * kHeadDim;
-            const float4 v = reinterpret_cast<const float4 *>(src)[lane];
-            bf16 *dst = vbase + (size_t)pos * kHeadDim;
-            reinterpret_cast<uint2 *>(dst)[lane] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
-        }
-        __threadfence_block();
-    }
-    __syncthreads();
-
-    // ---- Q fragments: row g8 (a query head, zero beyond G), contraction step s = 2c + e covers the head-dimension
-    //      elements 8 (4c + t4) + 4e + {0,1} (first half of the step) and + {2,3} (second half) ----
-    uint32_t qh[8][2], ql[8][2];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f), hi4 = lo4;
-        if (g8 < G) {
-            lo4 = *reinterpret_cast<const float4 *>(&qs[g8 < G ? g8 : 0][8 * (4 * c + t4)]);
-            hi4 = *reinterpret_cast<const float4 *>(&qs[g8 < G ? g8 : 0][8 * (4 * c + t4) + 4]);
-        }
-        split2(lo4.x, lo4.y, qh[2 * c][0], ql[2 * c][0]);
-        split2(lo4.z, lo4.w, qh[2 * c][1], ql[2 * c][1]);
-        split2(hi4.x, hi4.y, qh[2 * c + 1][0], ql[2 * c + 1][0]);
-        split2(hi4.z, hi4.w, qh[2 * c + 1][1], ql[2 * c + 1][1]);
-    }
-
-    float o[16][4];   // output tile j2: columns n = 2 t4, 2 t4 + 1 of row g8 in [0], [1]; [2], [3] belong to padding rows
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;   // per row g8 (identical across the 4 lanes of a row); l is a per-lane partial
-
-    for (int blk = warp; blk < n_blocks; blk += kWarps) {
-        const int p0 = c0 + blk * 16;
-        if (!(early && blk == warp)) load_block(p0);
-        // ---- scores: S[h] = Q K^T for the 8 positions of half h ----
-        float s[2][4];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            s[h][0] = s[h][1] = s[h][2] = s[h][3] = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t r0 = kf[h][c].x, r1 = kf[h][c].y, r2 = kf[h][c].z, r3 = kf[h][c].w;
-                mma_bf16(s[h], qh[2 * c][0], qh[2 * c][1], r0, r1);
-                mma_bf16(s[h], ql[2 * c][0], ql[2 * c][1], r0, r1);
-                mma_bf16(s[h], qh[2 * c + 1][0], qh[2 * c + 1][1], r2, r3);
-                mma_bf16(s[h], ql[2 * c + 1][0], ql[2 * c + 1][1], r2, r3);
-            }
-        }
-        // this lane holds row g8, positions p0 + 8h + 2 t4 + {0, 1}
-        float mx = -INFINITY;
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (p0 + 8 * h + 2 * t4 + e >= c1) s[h][e] = -INFINITY;
-                mx = fmaxf(mx, s[h][e]);
-            }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);           // finite: the block holds at least one valid position
-        const float alpha = exp2f(m_run - m_new);       // 0 on the first block
-        float pr[2][2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) pr[h][e] = exp2f(s[h][e] - m_new);
-        l_run = l_run * alpha + (pr[0][0] + pr[0][1] + pr[1][0] + pr[1][1]);
-        m_run = m_new;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
-        // ---- P fragments (contraction index = position inside the block), as value + residual ----
-        uint32_t ph0, pl0, ph1, pl1;
-        split2(pr[0][0], pr[0][1], ph0, pl0);   // positions 2 t4, 2 t4 + 1
-        split2(pr[1][0], pr[1][1], ph1, pl1);   // positions 2 t4 + 8, 2 t4 + 9
-        // ---- O += P V: output tile i covers head-dimension element (i < 8 ? 8 n + i : 64 + 8 n + i - 8), n = column ----
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int q2 = i >> 3, e = i & 7;
-            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
-            const uint32_t ra = (&vf[0][q2].x)[e >> 1], rb = (&vf[1][q2].x)[e >> 1];
-            const uint32_t rc = (&vf[2][q2].x)[e >> 1], rd = (&vf[3][q2].x)[e >> 1];
-            const uint32_t b0 = prmt(ra, rb, sel), b1 = prmt(rc, rd, sel);
-            mma_bf16(o[i], ph0, ph1, b0, b1);
-            mma_bf16(o[i], pl0, pl1, b0, b1);
-        }
-    }
-
-    NNC_TRACE_MARK2();
-    // ---- merge the warps: (o~, m, l) per query head into shared memory, then one partial per CTA ----
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (g8 < G) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int d0 = (i < 8) ? 8 * (2 * t4) + i : 64 + 8 * (2 * t4) + (i - 8);
-            comb[warp][g8][d0] = o[i][0];
-            comb[warp][g8][d0 + 8] = o[i][1];
-        }
-        if (t4 == 0) { comb[warp][g8][kHeadDim] = m_run; comb[warp][g8][kHeadDim + 1] = l_run; }
-    }
-    __syncthreads();
-
-    float *my_part = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits + split) * kPartStride;
-    // partial for head g lives at my_part + g * n_splits * kPartStride
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, comb[w][g][kHeadDim]);
-        float L = 0.f, acc = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const float sc = exp2f(comb[w][g][kHeadDim] - M);   // 0 for a warp that had no block
-            L = fmaf(sc, comb[w][g][kHeadDim + 1], L);
-            acc = fmaf(sc, comb[w][g][tid], acc);
-        }
-        float *pp = my_part + (size_t)g * p.n_splits * kPartStride;
-        pp[tid] = acc;
-        if (tid == 0) { pp[kHeadDim] = M; pp[kHeadDim + 1] = L; }
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned tk = atomicAdd(&p.tickets[b * p.nkv + j], 1u);
-        is_last = (tk == (unsigned)n_active - 1);
-    }
-    __syncthreads();
-    NNC_TRACE_MARK3();
-    if (!is_last) return;
-    __threadfence();
-    // ---- combine (last CTA of this sequence / KV head): o = sum_c 2^(m_c - M) o~_c / sum_c 2^(m_c - M) l_c.
-    //      Weights first (one warp per head, splits across lanes), then every thread folds its output element
-    //      over the splits with all loads of a batch of splits in flight at once. ----
-    float (*wgt)[kAttnMaxSplits] = reinterpret_cast<float (*)[kAttnMaxSplits]>(&comb[0][0][0]);   // [G][kAttnMaxSplits], reuses comb
-    __shared__ float inv_l[G];
-    const float *pbase = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits) * kPartStride;
-    for (int g = warp; g < G; g += kWarps) {
-        const float *pp = pbase + (size_t)g * p.n_splits * kPartStride;
-        float mv[2], lv[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int c = lane + 32 * u;
-            mv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim) : -INFINITY;
-            lv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim + 1) : 0.f;
-        }
-        const float M = warp_max(fmaxf(mv[0], mv[1]));
-        const float w0 = exp2f(mv[0] - M), w1 = exp2f(mv[1] - M);
-        wgt[g][lane] = w0;
-        wgt[g][lane + 32] = w1;
-        // fixed summation order over the splits: lane partials, then the shuffle tree
-        const float L = warp_sum(fmaf(w0, lv[0], w1 * lv[1]));
-        if (lane == 0) inv_l[g] = 1.f / L;
-    }
-    __syncthreads();
-    // one warp per head, 4 output elements per lane: 16-byte loads, a batch of splits in flight at once
-    for (int g = warp; g < G; g += kWarps) {
-        const float *pp = pbase + (size_t)g * p.n_splits * kPartStride + 4 * lane;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int cb = 0; cb < n_active; cb += 24) {
-            float4 v[24];
-#pragma unroll
-            for (int u = 0; u < 24; ++u)
-                v[u] = (cb + u < n_active) ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(cb + u) * kPartStride))
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 24; ++u) {
-                const float w = (cb + u < n_active) ? wgt[g][cb + u] : 0.f;
-                acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
-                acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
-            }
-        }
-        const float il = inv_l[g];
-        const float4 r = make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il);
-        const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + 4 * lane;
-        if (p.out_f32) *reinterpret_cast<float4 *>(p.out_f32 + oi) = r;
-        if (p.out_bf16) {
-            const uint2 hi = make_uint2(pack_bf16x2(r.x, r.y), pack_bf16x2(r.z, r.w));
-            *reinterpret_cast<uint2 *>(p.out_bf16 + oi) = hi;
-            if (p.out_bf16_lo)
-                *reinterpret_cast<uint2 *>(p.out_bf16_lo + oi) =
-                    make_uint2(pack_bf16x2(r.x - bf16_lo(hi.x), r.y - bf16_hi(hi.x)), pack_bf16x2(r.z - bf16_lo(hi.y), r.w - bf16_hi(hi.y)));
-        }
-    }
-    if (tid == 0) p.tickets[b * p.nkv + j] = 0u;
+    attn_decode_body<G, FUSED>(p, split, j, b, tid, sm, 1);
 }
+
 
 }  // namespace
 
@@ -386,7 +77,7 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
     p.nkv = nkv; p.max_seq = max_seq; p.n_splits = n_splits;
     p.g_q = fused ? fused->g_q : nullptr; p.g_k = fused ? fused->g_k : nullptr;
     p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;
-    dim3 grid(n_splits, nkv, batch), block(kWarps * 32);
+    dim3 grid(n_splits, nkv, batch), block(kAttnWarps * 32);
 #define NNC_ATTN_CASE(GG)                                                                  \
     case GG:                                                                               \
         return fused ? launch(lc, attn_decode_kernel<GG, true>, grid, block, p)           \

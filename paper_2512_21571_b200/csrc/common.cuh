@@ -80,11 +80,23 @@ struct TraceScope {
         }
     }
 };
+__device__ __forceinline__ unsigned long long trace_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+// free-standing record: [t0, t1] plus one extra interval end (mark = t_mark - t0)
+__device__ __forceinline__ void trace_event(unsigned kid, unsigned long long t0, unsigned long long t_mark, unsigned long long t1) {
+    if (!g_trace_buf) return;
+    unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+    const unsigned i = atomicAdd(g_trace_cnt, 1u);
+    if (i < kTraceMax) g_trace_buf[i] = TraceRec{kid, blockIdx.x, sm, (unsigned)(t_mark - t0), t0, t1, 0, 0, 0, 0};
+}
+#define NNC_TRACE_EVENT(kid, t0, tm, t1) trace_event(kid, t0, tm, t1)
+#define NNC_TRACE_NOW() trace_now()
 #define NNC_TRACE_SCOPE(kid) TraceScope nnc_trace_scope__(kid)
 #define NNC_TRACE_MARK() nnc_trace_scope__.set_mark()
 #define NNC_TRACE_MARK2() nnc_trace_scope__.set_mark2()
 #define NNC_TRACE_MARK3() nnc_trace_scope__.set_mark3()
 #else
+#define NNC_TRACE_EVENT(kid, t0, tm, t1)
+#define NNC_TRACE_NOW() 0ull
 #define NNC_TRACE_SCOPE(kid)
 #define NNC_TRACE_MARK()
 #define NNC_TRACE_MARK2()

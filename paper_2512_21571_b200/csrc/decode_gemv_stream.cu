@@ -447,6 +447,19 @@ bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int *ksplit_out, 
 
 }  // namespace
 
+bool gemv_stream_geometry(int n_out, int n_in, int sm_count, int mode, GemvGeom *out) {
+    if (!gemv_stream_supported(n_out, n_in, mode)) return false;
+    GemvGeom g;
+    g.n_out = n_out; g.K = n_in;
+    if (!pick_geometry(n_out, n_in, sm_count, mode == kGemvSwiglu, &g.ksplit, &g.rps)) return false;
+    g.kw = n_in / g.ksplit;
+    g.n_stages = (n_out + g.rps - 1) / g.rps;
+    const int j = (g.kw + 255) / 256;
+    g.J = j <= 4 ? j : (j <= 6 ? 6 : 8);
+    *out = g;
+    return true;
+}
+
 bool gemv_stream_supported(int n_out, int n_in, int mode) {
     int ks, rps;
     if (n_out < 1 || n_in % 8 || n_in < 64 || (mode == kGemvSwiglu && n_out % 2)) return false;

@@ -55,6 +55,42 @@ bool gemv_stream_supported(int n_out, int n_in, int mode);
 cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
                                const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr);
 
+// Slicing of one matrix for the streaming GEMV: consumer warps per row, columns per warp slice, rows per stage,
+// stages in the matrix, 16-byte chunks per lane per slice (rounded up to an instantiated value).
+struct GemvGeom {
+    int n_out, K;
+    int ksplit, kw, rps, n_stages, J;
+};
+bool gemv_stream_geometry(int n_out, int n_in, int sm_count, int mode, GemvGeom *out);
+
+// ---- whole-step decode kernel (decode_step_mega.cu) ----------------------------------------------------
+struct MegaLayer {
+    const bf16 *wqkv, *wo, *wgu, *wd, *g_in, *g_post, *g_q, *g_k;
+    bf16 *kc, *vc;
+};
+struct MegaParams {
+    const MegaLayer *layers;   // DEVICE array, n_layers entries
+    int n_layers;
+    GemvGeom gq, go, gg, gd, gl;   // QKV, O, gate/up, down, lm_head
+    const bf16 *embed, *lm_head, *g_final;
+    const int32_t *tokens;     // [1]
+    float *x, *qkv, *attn_out, *act, *logits;
+    ArgmaxScratch am;          // am.out == null: no arg-max
+    float *part;
+    uint32_t *tickets;
+    const int32_t *d_len;
+    const float *rope;
+    int nq, nkv, max_seq, n_splits, hidden, vocab;
+    float eps;
+    uint32_t *bars;            // 32 words of grid-barrier state (counters, release word, abort word), zero at launch
+    int *status;
+    int stages;                // ring depth
+    uint32_t slot_bytes;       // ring slot size (largest stage of the step)
+};
+// false: shape outside what the whole-step kernel covers (the caller uses the kernel-per-phase path)
+bool decode_mega_supported(const MegaParams &p, int sm_count);
+cudaError_t launch_decode_mega(const LaunchCtx &lc, const MegaParams &p);
+
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
                          int vocab, float *tap);
