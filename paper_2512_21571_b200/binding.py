@@ -71,6 +71,8 @@ EXPORTS = {
     "nnc_attn_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
     "nnc_op_attn_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "nnc_op_attn_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                      C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "nnc_op_attn_decode_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
 }
@@ -310,3 +312,15 @@ def op_gemm_splitk(X: torch.Tensor, W: torch.Tensor, scratch: torch.Tensor, out_
                                int(accumulate_into is not None), scratch.data_ptr(), scratch.numel(), _stream_ptr()),
         "nnc_op_gemm_splitk")
     return Y
+
+
+def op_attn_prefill(qkv: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tensor, T: int, n_q_heads: int, n_past: int):
+    """nnc_op_attn_prefill; returns (out, out_lo), bf16 [batch * T][n_q_heads * 128]."""
+    batch, nkv, max_seq, _ = kcache.shape
+    out = torch.empty(batch * T, n_q_heads * 128, dtype=torch.bfloat16, device="cuda")
+    out_lo = torch.empty_like(out)
+    past = torch.tensor([n_past], dtype=torch.int32, device="cuda")
+    _ok(lib.nnc_op_attn_prefill(_dev(qkv, torch.float32), _dev(kcache, torch.bfloat16), _dev(vcache, torch.bfloat16),
+                                out.data_ptr(), out_lo.data_ptr(), batch, T, n_q_heads, nkv, max_seq, past.data_ptr(),
+                                _stream_ptr()), "nnc_op_attn_prefill")
+    return out, out_lo

@@ -795,4 +795,16 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 
+int nnc_op_attn_prefill(const float *qkv, const void *kcache, const void *vcache, void *out, void *out_lo, int32_t batch,
+                        int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, const int32_t *n_past_dev,
+                        void *cuda_stream) {
+    if (!qkv || !kcache || !vcache || !out || !n_past_dev) return NNC_ERR_INVALID_ARG;
+    if (batch <= 0 || T <= 0 || n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % n_kv_heads || max_seq < T) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, (const bf16 *)kcache, (const bf16 *)vcache, (bf16 *)out,
+                                        (bf16 *)out_lo, n_q_heads, n_kv_heads, max_seq, n_past_dev);
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
 }  // extern "C"

@@ -169,3 +169,27 @@ def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
     assert (Y3.double() - (acc.double() + ref)).abs().max().item() < 1e-4 * math.sqrt(K)
     Yb = nnc.op_gemm_splitk(hi, W, scratch, out_f32=False)
     assert torch.allclose(Yb.float(), ref.float(), rtol=2e-2, atol=2e-2)
+
+
+@pytest.mark.parametrize("batch,T,nq,nkv,n_past", [(1, 19, 2, 1, 0), (2, 130, 4, 2, 7), (1, 300, 8, 2, 0), (1, 64, 16, 8, 200)])
+def test_attn_prefill_against_oracle(nnc, oracle_mod, batch, T, nq, nkv, n_past):
+    """Causal prompt-phase attention: query s sees cache positions 0 .. n_past + s.  Rows are checked against the
+    oracle's single-query attention over the matching cache prefix (sampled rows, all heads of those rows)."""
+    max_seq = n_past + T + 5
+    heads = nq + 2 * nkv
+    qkv = synth.normal(9, 1, (batch * T, heads * 128), 1.0, torch.float32, "cuda")
+    kc = synth.normal(9, 2, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    vc = synth.normal(9, 3, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    kc[:, :, n_past + T:] = float("nan"); vc[:, :, n_past + T:] = float("nan")   # never to be read into a result
+    out, out_lo = nnc.op_attn_prefill(qkv, kc, vc, T, nq, n_past)
+    torch.cuda.synchronize()
+    got = (out.float() + out_lo.float()).cpu().view(batch, T, nq, 128)
+    assert torch.isfinite(got).all()
+    G = nq // nkv
+    qc, kcc, vcc = qkv.cpu().view(batch, T, heads, 128), kc.cpu(), vc.cpu()
+    for b in range(batch):
+        for s in sorted(set([0, 1, T // 2, T - 1, min(T - 1, 127), min(T - 1, 128)])):
+            n = n_past + s + 1
+            for h in range(nq):
+                want = oracle_mod.attend(qc[b, s, h].contiguous(), kcc[b, h // G, :n].contiguous(), vcc[b, h // G, :n].contiguous())
+                assert torch.allclose(got[b, s, h], want, rtol=1e-3, atol=1e-4), (b, s, h)
