@@ -39,7 +39,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(const Attn
         const int c0 = split * chunk, c1 = min(c0 + chunk, min(n_guess, p.max_seq));
         if (tid < 2 && c1 > c0) {
             const bf16 *src = (tid ? p.vcache : p.kcache) + head_off + (size_t)c0 * kHeadDim;
-            const uint32_t bytes = (uint32_t)(c1 - c0) * kHeadDim * 2u;
+            // short ranges whole; long ranges only their head (the body prefetches ahead of itself as it goes)
+            const uint32_t bytes = (uint32_t)min(c1 - c0, kPrefetchAhead * kAttnWarps * 16) * kHeadDim * 2u;
             asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
         }
     }

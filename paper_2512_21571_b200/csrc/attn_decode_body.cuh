@@ -9,6 +9,7 @@ namespace nnc {
 
 constexpr int kPartStride = kHeadDim + 4;  // o~[128], m, l, 2 pad words (rows stay 16-byte aligned)
 constexpr int kAttnWarps = 4;
+constexpr int kPrefetchAhead = 6;   // blocks of 16 positions, per warp
 
 __device__ __forceinline__ uint4 ldg_cg(const void *p) {
     uint4 v;
@@ -184,6 +185,15 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     for (int blk = warp; blk < n_blocks; blk += kWarps) {
         const int p0 = c0 + blk * 16;
         if (!(early && blk == warp)) load_block(p0);
+        // long ranges: ask L2 for the block this warp will reach kPrefetchAhead iterations from now (16 rows of K and
+        // of V, 4 KB each, contiguous), so that the fragment loads above find their rows in L2
+        {
+            const int pf = p0 + kPrefetchAhead * kWarps * 16;
+            if (lane < 2 && pf + 16 <= c1) {
+                const bf16 *src = (lane ? vbase : kbase) + (size_t)pf * kHeadDim;
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(16u * kHeadDim * 2u) : "memory");
+            }
+        }
         // ---- scores: S[h] = Q K^T for the 8 positions of half h ----
         float s[2][4];
 #pragma unroll
