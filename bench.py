@@ -529,7 +529,8 @@ def main():
 
     line = {"metric": metric_name(wl), "value": round(value, 2), "unit": "tokens/s", "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": round(ms / steps, 4), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 weights and cache, f32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "dtype_detail": "bf16 weights and KV cache, fp32 activations and accumulation",
+            "data": "synthetic",
             "config": config_of(wl), "clocks": clocks,
             "e2e": {"value": round(e2e_value, 2), "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": round(ms_e / steps, 4)},

@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(const Attn
         int chunk = (n_guess + p.n_splits - 1) / p.n_splits;
         chunk = (chunk + 15) & ~15;
         if (chunk < 16) chunk = 16;
+        if (n_guess <= kSingleRange) chunk = kSingleRange;
         const int c0 = split * chunk, c1 = min(c0 + chunk, min(n_guess, p.max_seq));
         if (tid < 2 && c1 > c0) {
             const bf16 *src = (tid ? p.vcache : p.kcache) + head_off + (size_t)c0 * kHeadDim;

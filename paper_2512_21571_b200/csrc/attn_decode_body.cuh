@@ -9,6 +9,7 @@ namespace nnc {
 
 constexpr int kPartStride = kHeadDim + 4;  // o~[128], m, l, 2 pad words (rows stay 16-byte aligned)
 constexpr int kAttnWarps = 4;
+constexpr int kSingleRange = 128;    // contexts up to this length are handled by one CTA per KV head
 constexpr int kPrefetchAhead = 6;   // blocks of 16 positions, per warp
 
 __device__ __forceinline__ uint4 ldg_cg(const void *p) {
@@ -98,6 +99,7 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     int chunk = (n_ctx + p.n_splits - 1) / p.n_splits;
     chunk = (chunk + 15) & ~15;
     if (chunk < 16) chunk = 16;
+    if (n_ctx <= kSingleRange) chunk = kSingleRange;   // short context: one CTA per KV head, no partials
     const int c0 = split * chunk;
     const int c1 = min(c0 + chunk, n_ctx);
     const int n_active = (n_ctx + chunk - 1) / chunk;
@@ -275,10 +277,23 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
             L = fmaf(sc, sm.comb[w][g][kHeadDim + 1], L);
             acc = fmaf(sc, sm.comb[w][g][tid], acc);
         }
+        if (n_active == 1) {
+            // the only range of this head: no partial, no ticket -- the same arithmetic the combine would do
+            const float r = acc * (1.f / L);
+            const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + tid;
+            if (p.out_f32) p.out_f32[oi] = r;
+            if (p.out_bf16) {
+                const bf16 hi = __float2bfloat16_rn(r);
+                p.out_bf16[oi] = hi;
+                if (p.out_bf16_lo) p.out_bf16_lo[oi] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            }
+            continue;
+        }
         float *pp = my_part + (size_t)g * p.n_splits * kPartStride;
         pp[tid] = acc;
         if (tid == 0) { pp[kHeadDim] = M; pp[kHeadDim + 1] = L; }
     }
+    if (n_active == 1) return;
     __threadfence();
     attn_group_sync(bar_id);
     if (tid == 0) {
