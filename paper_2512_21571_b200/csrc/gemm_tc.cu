@@ -208,6 +208,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 NNC_UNIT_DECODE(tile)
                 const int w_row = SWAP ? mt * kBM : nt * BN;
                 const int x_row = SWAP ? nt * BN : mt * kBM;
+                const unsigned long long tr0 = NNC_TRACE_NOW();
+                (void)tr0;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     mbar_expect_tx(full_bar(stage), L::kStage);
@@ -222,6 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
+                if (blockIdx.x == 0) NNC_TRACE_EVENT(201, tr0, tr0, NNC_TRACE_NOW());
             }
         }
     } else if (warp == 1) {
@@ -234,6 +237,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                const unsigned long long tr0 = NNC_TRACE_NOW();
+                (void)tr0;
                 NNC_UNIT_DECODE(tile)
                 (void)mt; (void)nt;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
@@ -263,6 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 if (!ok) break;
                 umma_commit(tfull_bar(acc));
+                if (blockIdx.x == 0) NNC_TRACE_EVENT(202, tr0, tr0, NNC_TRACE_NOW());
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -307,6 +313,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (!got && !(SWAP && p.ksplit > 1)) break;
             tc_fence_after();
             const int m = mt * kBM + quarter * 32 + lane;  // D row held by this thread
+            const unsigned long long tr0 = NNC_TRACE_NOW();
+            unsigned long long tr1 = tr0;
+            (void)tr0; (void)tr1;
             if (SWAP && p.ksplit > 1) {
                 // ---- split K: park this piece's fp32 tile, take a ticket; the piece that arrives last adds the
                 //      pieces in piece order and runs the epilogue (nobody waits) ----
@@ -325,6 +334,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(acc));
                 }
+                tr1 = NNC_TRACE_NOW();
                 __threadfence();
                 asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (*abort_flag) break;
@@ -368,6 +378,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                 }
                 asm volatile("bar.sync 2, 128;" ::: "memory");   // split_last is rewritten by the next unit
+                if (blockIdx.x == 0 && warp == 2 && lane == 0) NNC_TRACE_EVENT(203, tr0, tr1, NNC_TRACE_NOW());
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 continue;
             }

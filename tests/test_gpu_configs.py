@@ -104,3 +104,64 @@ def test_config5_mode1_qwen3_8b_prefill_sampled(oracle_mod):
     # batched prefill on the 8B shape; the oracle's share is one sequence of 256 tokens (the full 4 x 2048 is
     # ~114 TFLOP of CPU work); batch independence is covered by test_batched_sequences_are_independent
     _run(oracle_mod, "qwen3-8b", 4, prefill=int(os.environ.get("NNC_TEST_PREFILL", "256")), decode=STEPS or 2)
+
+
+def test_config5_mode2_qwen3_8b_batch32_ctx8192_sampled(oracle_mod):
+    """Batched decode on the 8B shape: 32 sequences with 8192 cached positions each, two lock-step decode steps
+    through the tensor-core path.  The oracle's share: two of the 32 sequences (the first and one in the middle),
+    each with its own imported cache; the rest is covered by the batch-independence property on a small shape."""
+    name, seed, B, ctx, steps = "qwen3-8b", 4, int(os.environ.get("NNC_TEST_BATCH", "32")), 8192, 2
+    shape = synth.SHAPES[name]
+    m, o, w = make_pair(oracle_mod, shape, seed, max_seq=ctx + steps + 1, max_batch=B, max_tokens=B)
+    for b in range(B):
+        for l in range(shape.n_layers):
+            k, v = synth.kv_fill(shape, seed + 1000, l, ctx, device="cuda", batch_index=b)
+            m.kv_import(l, b, k, v)
+    m.set_length(ctx)
+    toks = torch.stack([synth.tokens(seed + 2000, b, steps, shape.vocab) for b in range(B)], 1).cuda()   # [steps][B]
+    got = []
+    logits = torch.empty(B, shape.vocab, device="cuda")
+    for s in range(steps):
+        m.decode_step(toks[s].contiguous(), logits)
+        got.append(logits.cpu().clone())
+    assert m.device_status() == 0
+    worst = 0.0
+    for b in sorted(set([0, B // 2 + 1 if B > 2 else B - 1])):
+        o.reset()
+        for l in range(shape.n_layers):
+            k, v = synth.kv_fill(shape, seed + 1000, l, ctx, device="cuda", batch_index=b)
+            o.kv_import(l, k.cpu(), v.cpu())
+        for s in range(steps):
+            lo, _ = o.forward(toks[s, b:b + 1].cpu())
+            err = (got[s][b] - lo).abs().max().item()
+            worst = max(worst, err)
+            idx, margin = oracle_mod.argmax_margin(lo)
+            if margin > MARGIN:
+                assert int(got[s][b].argmax()) == idx, (b, s)
+    _log(f"{name} batched decode B={B} ctx {ctx}, {steps} steps: logits max-abs {worst:.3e} on 2 sampled sequences")
+    assert worst < LOGIT_TOL
+    m.close(); o.close()
+
+
+def test_config5_mode1_full_size_batch_independence(oracle_mod):
+    """The launch configuration the benchmark times (8B shape, 4 x 2048 tokens): every sequence of the batched call
+    must equal the same sequence run alone (logits and appended cache rows), which ties the full-size batched call to
+    the single-sequence path that the oracle checks on a 256-token prefix."""
+    name, seed, B, T = "qwen3-8b", 4, 4, 2048
+    shape = synth.SHAPES[name]
+    m, o, w = make_pair(oracle_mod, shape, seed, max_seq=T, max_batch=B, max_tokens=B * T)
+    o.close()
+    toks = torch.stack([synth.prompt_tokens(shape, seed + 1000, T, batch_index=b) for b in range(B)]).cuda()
+    lg = m.prefill(toks).clone()
+    kv_batched = [m.kv_export(l, 2, T) for l in (0, shape.n_layers - 1)]
+    assert torch.isfinite(lg).all()
+    for b in (2,):
+        m.set_length(0)
+        l1 = m.prefill(toks[b:b + 1].contiguous())
+        # sequence b alone lands in cache slot 0; same tiles, same order of accumulation inside a sequence
+        assert (l1[0] - lg[b]).abs().max().item() < 1e-3, b
+        for (kb, vb), l in zip(kv_batched, (0, shape.n_layers - 1)):
+            k1, v1 = m.kv_export(l, 0, T)
+            assert (k1.float() - kb.float()).abs().max().item() < 2e-2 and (v1.float() - vb.float()).abs().max().item() < 2e-2
+    assert m.device_status() == 0
+    m.close()
