@@ -190,6 +190,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    // launched with programmatic stream serialization: the set-up above overlaps the previous kernel's tail, and the
+    // next kernel may start its own set-up now; everything that touches that kernel's data waits below
+    pdl_launch_dependents();
 
     const int kb_count = p.K / (kBK * KA);   // pipeline stages along K
     const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;   // work units: (output tile, K piece)
@@ -201,6 +204,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
+            pdl_wait();
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -274,6 +278,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else {  // ---------------- epilogue warps 2..5 ----------------
         const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+        pdl_wait();
         int acc = 0;
         uint32_t acc_phase = 0;
         // SWAP stores: row m = weight row, columns = tokens n0 .. n0 + 31; a warp stores 32 consecutive weight rows per token
@@ -554,8 +559,17 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
     int grid = p.m_tiles * p.n_tiles * p.ksplit;
     if (grid > lc.sm_count) grid = lc.sm_count;
     if (lc.launches) ++*lc.launches;
-    kern<<<grid, kGemmThreads, L::kBytes, lc.stream>>>(map_w, map_x, map_x_lo, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = L::kBytes;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, map_w, map_x, map_x_lo, p);
 }
 
 // Few tokens (weights on the M side): a stage carries 4 (<= 32 tokens) or 2 (<= 64) consecutive K slabs, so that

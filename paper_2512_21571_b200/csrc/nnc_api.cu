@@ -216,7 +216,7 @@ int decode_b1_mega_launches(nnc_model *m, const int32_t *tokens, float *logits, 
 int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float *logits, int all_positions) {
     const nnc_config &c = m->c;
     const int R = batch * T, H = c.hidden, I = c.intermediate, qd = m->qd(), qkvd = m->qkvd();
-    LaunchCtx lc = ctx(m, false);
+    LaunchCtx lc = ctx(m, m->pdl);
     NNC_CUDA(m, launch_embed(lc, m->embed, tokens, m->xt, R, H, c.vocab, m->taps));
     const int n_splits = attn_decode_splits(m->sm_count, batch, c.n_kv_heads, c.max_seq);
     for (int l = 0; l < c.n_layers; ++l) {
