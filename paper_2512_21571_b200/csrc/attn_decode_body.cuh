@@ -18,12 +18,19 @@ __device__ __forceinline__ uint4 ldg_cg(const void *p) {
     return v;
 }
 
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-    // rows 8..15 of the 16-row operand are padding: a1 = a3 = 0
+__device__ __forceinline__ void mma_bf16_full(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// transposes an 8x8 matrix of 16-bit elements held one row per 4 lanes (lane l: row l / 4, columns 2 (l % 4), + 1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t r;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(x));
+    return r;
 }
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -107,8 +114,9 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
 
     // ---- K/V fragment loads of one block of 16 positions: K rows p0 + 8h + g8 (h = 0, 1), V rows
     //      p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9}; rows past the range are clamped here and masked later ----
-    uint4 kf[2][4], vf[4][2];
-    auto load_block = [&](int p0) {
+    // two register buffers: the warp's next block is in flight while it works on the current one
+    uint4 kfa[2][4], vfa[4][2], kfb[2][4], vfb[4][2];
+    auto load_block = [&](uint4 (&kf)[2][4], uint4 (&vf)[4][2], int p0) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int pos = min(p0 + 8 * h + g8, c1 - 1);
@@ -128,7 +136,7 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     // the warp's first block is requested now and lands while the queries are prepared -- unless it holds the row
     // that is appended below
     const bool early = warp < n_blocks && !(FUSED && c0 + warp * 16 + 16 >= n_ctx);
-    if (early) load_block(c0 + warp * 16);
+    if (early) load_block(kfa, vfa, c0 + warp * 16);
 
     // ---- queries (and, fused, the new token's K/V row) ----
     const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);   // scores in log2 units
@@ -163,8 +171,9 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     }
     attn_group_sync(bar_id);
 
-    // ---- Q fragments: row g8 (a query head, zero beyond G), contraction step s = 2c + e covers the head-dimension
-    //      elements 8 (4c + t4) + 4e + {0,1} (first half of the step) and + {2,3} (second half) ----
+    // ---- Q^T fragments (the 8-column operand): column g8 is a query head (zero beyond G); contraction step
+    //      s = 2c + e covers the head-dimension elements 8 (4c + t4) + 4e + {0,1} (first half of the step) and
+    //      + {2,3} (second half), the same elements the K chunk c of this lane holds ----
     uint32_t qh[8][2], ql[8][2];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -179,14 +188,15 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
         split2(hi4.z, hi4.w, qh[2 * c + 1][1], ql[2 * c + 1][1]);
     }
 
-    float o[16][4];   // output tile j2: columns n = 2 t4, 2 t4 + 1 of row g8 in [0], [1]; [2], [3] belong to padding rows
+    // O^T tile i: rows are head-dimension elements 8 g8 + i ([0], [1]) and 64 + 8 g8 + i ([2], [3]); columns are the
+    // query heads 2 t4 ([0], [2]) and 2 t4 + 1 ([1], [3])
+    float o[8][4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;   // per row g8 (identical across the 4 lanes of a row); l is a per-lane partial
+    for (int i = 0; i < 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    // per head 2 t4 + e: running maximum (identical across the 8 lanes that share t4) and this lane's partial sum
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
-    for (int blk = warp; blk < n_blocks; blk += kWarps) {
-        const int p0 = c0 + blk * 16;
-        if (!(early && blk == warp)) load_block(p0);
+    auto process_block = [&](const uint4 (&kf)[2][4], const uint4 (&vf)[4][2], int p0) {
         // long ranges: ask L2 for the block this warp will reach kPrefetchAhead iterations from now (16 rows of K and
         // of V, 4 KB each, contiguous), so that the fragment loads above find their rows in L2
         {
@@ -196,70 +206,86 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
                 asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(16u * kHeadDim * 2u) : "memory");
             }
         }
-        // ---- scores: S[h] = Q K^T for the 8 positions of half h ----
-        float s[2][4];
+        // ---- scores, transposed: S^T = K Q^T; s[0], s[1] = position p0 + g8, heads 2 t4, 2 t4 + 1;
+        //      s[2], s[3] = position p0 + 8 + g8 ----
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            s[h][0] = s[h][1] = s[h][2] = s[h][3] = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t r0 = kf[h][c].x, r1 = kf[h][c].y, r2 = kf[h][c].z, r3 = kf[h][c].w;
-                mma_bf16(s[h], qh[2 * c][0], qh[2 * c][1], r0, r1);
-                mma_bf16(s[h], ql[2 * c][0], ql[2 * c][1], r0, r1);
-                mma_bf16(s[h], qh[2 * c + 1][0], qh[2 * c + 1][1], r2, r3);
-                mma_bf16(s[h], ql[2 * c + 1][0], ql[2 * c + 1][1], r2, r3);
-            }
+        for (int c = 0; c < 4; ++c) {
+            mma_bf16_full(s, kf[0][c].x, kf[1][c].x, kf[0][c].y, kf[1][c].y, qh[2 * c][0], qh[2 * c][1]);
+            mma_bf16_full(s, kf[0][c].x, kf[1][c].x, kf[0][c].y, kf[1][c].y, ql[2 * c][0], ql[2 * c][1]);
+            mma_bf16_full(s, kf[0][c].z, kf[1][c].z, kf[0][c].w, kf[1][c].w, qh[2 * c + 1][0], qh[2 * c + 1][1]);
+            mma_bf16_full(s, kf[0][c].z, kf[1][c].z, kf[0][c].w, kf[1][c].w, ql[2 * c + 1][0], ql[2 * c + 1][1]);
         }
-        // this lane holds row g8, positions p0 + 8h + 2 t4 + {0, 1}
-        float mx = -INFINITY;
+        if (p0 + g8 >= c1) s[0] = s[1] = -INFINITY;
+        if (p0 + 8 + g8 >= c1) s[2] = s[3] = -INFINITY;
+        float pr[4], alpha[2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+        for (int e = 0; e < 2; ++e) {
+            float mx = fmaxf(s[e], s[e + 2]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float m_new = fmaxf(m_run[e], mx);        // finite: the block holds at least one valid position
+            alpha[e] = exp2f(m_run[e] - m_new);             // 0 on the first block
+            pr[e] = exp2f(s[e] - m_new);
+            pr[e + 2] = exp2f(s[e + 2] - m_new);
+            l_run[e] = l_run[e] * alpha[e] + (pr[e] + pr[e + 2]);
+            m_run[e] = m_new;
+        }
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (p0 + 8 * h + 2 * t4 + e >= c1) s[h][e] = -INFINITY;
-                mx = fmaxf(mx, s[h][e]);
-            }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);           // finite: the block holds at least one valid position
-        const float alpha = exp2f(m_run - m_new);       // 0 on the first block
-        float pr[2][2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) pr[h][e] = exp2f(s[h][e] - m_new);
-        l_run = l_run * alpha + (pr[0][0] + pr[0][1] + pr[1][0] + pr[1][1]);
-        m_run = m_new;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
-        // ---- P fragments (contraction index = position inside the block), as value + residual ----
+        for (int i = 0; i < 8; ++i) { o[i][0] *= alpha[0]; o[i][1] *= alpha[1]; o[i][2] *= alpha[0]; o[i][3] *= alpha[1]; }
+        // ---- P^T fragments (contraction index = position inside the block), as value + residual: the 8x8 blocks
+        //      (position, head) this lane holds a row of are transposed across the warp, after which this lane holds
+        //      head g8, positions 2 t4, 2 t4 + 1 (first block) and 2 t4 + 8, 2 t4 + 9 (second block) ----
         uint32_t ph0, pl0, ph1, pl1;
-        split2(pr[0][0], pr[0][1], ph0, pl0);   // positions 2 t4, 2 t4 + 1
-        split2(pr[1][0], pr[1][1], ph1, pl1);   // positions 2 t4 + 8, 2 t4 + 9
-        // ---- O += P V: output tile i covers head-dimension element (i < 8 ? 8 n + i : 64 + 8 n + i - 8), n = column ----
+        split2(pr[0], pr[1], ph0, pl0);
+        split2(pr[2], pr[3], ph1, pl1);
+        ph0 = movmatrix_trans(ph0); pl0 = movmatrix_trans(pl0);
+        ph1 = movmatrix_trans(ph1); pl1 = movmatrix_trans(pl1);
+        // ---- O^T += V^T P^T ----
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int q2 = i >> 3, e = i & 7;
-            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
-            const uint32_t ra = (&vf[0][q2].x)[e >> 1], rb = (&vf[1][q2].x)[e >> 1];
-            const uint32_t rc = (&vf[2][q2].x)[e >> 1], rd = (&vf[3][q2].x)[e >> 1];
-            const uint32_t b0 = prmt(ra, rb, sel), b1 = prmt(rc, rd, sel);
-            mma_bf16(o[i], ph0, ph1, b0, b1);
-            mma_bf16(o[i], pl0, pl1, b0, b1);
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t sel = (i & 1) ? 0x7632u : 0x5410u;
+            const uint32_t a0 = prmt((&vf[0][0].x)[i >> 1], (&vf[1][0].x)[i >> 1], sel);
+            const uint32_t a1 = prmt((&vf[0][1].x)[i >> 1], (&vf[1][1].x)[i >> 1], sel);
+            const uint32_t a2 = prmt((&vf[2][0].x)[i >> 1], (&vf[3][0].x)[i >> 1], sel);
+            const uint32_t a3 = prmt((&vf[2][1].x)[i >> 1], (&vf[3][1].x)[i >> 1], sel);
+            mma_bf16_full(o[i], a0, a1, a2, a3, ph0, ph1);
+            mma_bf16_full(o[i], a0, a1, a2, a3, pl0, pl1);
+        }
+    };
+    {
+        int blk = warp;
+        if (blk < n_blocks && !early) load_block(kfa, vfa, c0 + blk * 16);
+        while (blk < n_blocks) {
+            if (blk + kWarps < n_blocks) load_block(kfb, vfb, c0 + (blk + kWarps) * 16);
+            process_block(kfa, vfa, c0 + blk * 16);
+            blk += kWarps;
+            if (blk >= n_blocks) break;
+            if (blk + kWarps < n_blocks) load_block(kfa, vfa, c0 + (blk + kWarps) * 16);
+            process_block(kfb, vfb, c0 + blk * 16);
+            blk += kWarps;
         }
     }
 
     // ---- merge the warps: (o~, m, l) per query head into shared memory, then one partial per CTA ----
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (g8 < G) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int d0 = (i < 8) ? 8 * (2 * t4) + i : 64 + 8 * (2 * t4) + (i - 8);
-            sm.comb[warp][g8][d0] = o[i][0];
-            sm.comb[warp][g8][d0 + 8] = o[i][1];
+    for (int e = 0; e < 2; ++e) {
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+    }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int head = 2 * t4 + e;
+        if (head < G) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                sm.comb[warp][head][8 * g8 + i] = o[i][e];
+                sm.comb[warp][head][64 + 8 * g8 + i] = o[i][2 + e];
+            }
+            if (g8 == 0) { sm.comb[warp][head][kHeadDim] = m_run[e]; sm.comb[warp][head][kHeadDim + 1] = l_run[e]; }
         }
-        if (t4 == 0) { sm.comb[warp][g8][kHeadDim] = m_run; sm.comb[warp][g8][kHeadDim + 1] = l_run; }
     }
     attn_group_sync(bar_id);
 
