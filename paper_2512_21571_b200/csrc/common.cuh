@@ -53,6 +53,9 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // Every CTA appends {kernel id, block, SM, start, end} (globaltimer ns) to a device buffer when it exits;
 // nnc_trace_dump() copies the buffer to the host.  Compiled out of the normal library.  Each translation unit
 // holds its own copy of the two pointers (no relocatable device code) and registers a binder for them.
+#ifndef NNC_TRACE_ALL_CTAS
+#define NNC_TRACE_ALL_CTAS 0   // tracing builds may record per-unit events of every CTA instead of CTA 0's only
+#endif
 #ifdef NNC_TRACE
 struct TraceRec { unsigned kid, block, smid, mark; unsigned long long t0, t1; unsigned mark2, mark3, pad0, pad1; };
 constexpr unsigned kTraceMax = 1u << 20;

@@ -129,10 +129,58 @@ struct GemmParams {
     int T, N, K;      // tokens, weight rows, reduction
     int ldy;          // output row stride in elements
     int m_tiles, n_tiles;
-    int ksplit;          // K is cut into ksplit pieces per output tile (SWAP only); 1 = no split
-    float *part;         // ksplit > 1: fp32 partial tiles [tile][piece][BN / 32][128 rows][32]
-    uint32_t *tickets;   // ksplit > 1: one arrival counter per output tile, zero at rest
+    int stream;          // 1: the (tile, K stage) space is cut into one contiguous range per CTA (SWAP only)
+    float *part;         // stream: fp32 partial tiles [CTA][first / last segment][BN / 32][8][128 rows][4]
+    uint32_t *tickets;   // stream: one arrival counter per output tile, zero at rest
     int *status;
+};
+
+// One piece of work: K stages [kb_lo, kb_hi) of output tile tile_id.  n_pieces > 1: the tile's K range is shared by
+// n_pieces consecutive CTAs, this one holding piece number `piece` (pieces are numbered in K order).
+struct Segment {
+    int tile_id, kb_lo, kb_hi, piece, n_pieces, first_cta;
+};
+
+// Enumerates a CTA's segments; every role of the CTA walks the same list.
+//   classic: whole tiles, strided over the grid.
+//   stream:  the tile-major list of all (tile, K stage) pairs is cut into gridDim.x equal contiguous ranges, so every
+//            CTA streams the same number of weight bytes whatever the tile count; a tile whose stages fall into
+//            several ranges is finished by whichever of those CTAs gets there last (see the epilogue).
+struct WorkIter {
+    int kb_count, tiles, stream;
+    long long total;   // stream: tiles * kb_count
+    long long s, s_begin, s_end;
+    __device__ long long range_lo(int cta) const { return (long long)cta * total / (long long)gridDim.x; }
+    __device__ int cta_of(long long stage) const { return (int)(((stage + 1) * (long long)gridDim.x - 1) / total); }
+    __device__ WorkIter(int tiles_, int kb_count_, int stream_) : kb_count(kb_count_), tiles(tiles_), stream(stream_) {
+        total = (long long)tiles * kb_count;
+        if (stream) { s_begin = range_lo(blockIdx.x); s_end = range_lo(blockIdx.x + 1); }
+        else { s_begin = blockIdx.x; s_end = tiles; }
+        s = s_begin;
+    }
+    __device__ bool next(Segment &g) {
+        if (s >= s_end) return false;
+        if (!stream) {
+            g = Segment{(int)s, 0, kb_count, 0, 1, (int)blockIdx.x};
+            s += gridDim.x;
+            return true;
+        }
+        const int tile = (int)(s / kb_count);
+        const long long t0 = (long long)tile * kb_count;
+        const int kb_lo = (int)(s - t0);
+        const long long left = s_end - s;
+        const int len = (kb_count - kb_lo < left) ? kb_count - kb_lo : (int)left;
+        const int c_first = cta_of(t0), c_last = cta_of(t0 + kb_count - 1);
+        g = Segment{tile, kb_lo, kb_lo + len, (int)blockIdx.x - c_first, c_last - c_first + 1, c_first};
+        s += len;
+        return true;
+    }
+    // partial-tile slot of the piece CTA `cta` holds of tile `tile`: a CTA has at most two partial segments, the
+    // first of its range (slot 0) and the last (slot 1)
+    __device__ int slot_of(int cta, int tile) const {
+        const long long lo = range_lo(cta), t0 = (long long)tile * kb_count;
+        return 2 * cta + ((lo >= t0) ? 0 : 1);
+    }
 };
 
 // Shared-memory stage: [weight tile][activation tile][activation residual tile (SPLIT)].
@@ -195,12 +243,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     pdl_launch_dependents();
 
     const int kb_count = p.K / (kBK * KA);   // pipeline stages along K
-    const int total_tiles = p.m_tiles * p.n_tiles * p.ksplit;   // work units: (output tile, K piece)
-    // unit u -> output tile u / ksplit (m fastest), K blocks [kb_lo, kb_hi)
-#define NNC_UNIT_DECODE(u)                                                        \
-    const int tile_id = (u) / p.ksplit, ks_id = (u) % p.ksplit;                   \
-    const int mt = tile_id % p.m_tiles, nt = tile_id / p.m_tiles;                 \
-    const int kb_lo = ks_id * kb_count / p.ksplit, kb_hi = (ks_id + 1) * kb_count / p.ksplit;
+    const int total_tiles = p.m_tiles * p.n_tiles;   // output tile id: m fastest
+    const int stream = SWAP ? p.stream : 0;
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
@@ -208,8 +252,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                NNC_UNIT_DECODE(tile)
+            WorkIter it(total_tiles, kb_count, stream);
+            Segment g;
+            while (ok && it.next(g)) {
+                const int mt = g.tile_id % p.m_tiles, nt = g.tile_id / p.m_tiles;
+                const int kb_lo = g.kb_lo, kb_hi = g.kb_hi;
                 const int w_row = SWAP ? mt * kBM : nt * BN;
                 const int x_row = SWAP ? nt * BN : mt * kBM;
                 const unsigned long long tr0 = NNC_TRACE_NOW();
@@ -228,7 +275,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (blockIdx.x == 0) NNC_TRACE_EVENT(201, tr0, tr0, NNC_TRACE_NOW());
+                if (NNC_TRACE_ALL_CTAS || blockIdx.x == 0) NNC_TRACE_EVENT(201, tr0, tr0, NNC_TRACE_NOW());
             }
         }
     } else if (warp == 1) {
@@ -237,16 +284,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            WorkIter it(total_tiles, kb_count, stream);
+            Segment g;
+            while (ok && it.next(g)) {
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 const unsigned long long tr0 = NNC_TRACE_NOW();
-                (void)tr0;
-                NNC_UNIT_DECODE(tile)
-                (void)mt; (void)nt;
+                unsigned long long tr_first = tr0;
+                (void)tr0; (void)tr_first;
+                const int kb_lo = g.kb_lo, kb_hi = g.kb_hi;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    if (kb == kb_lo) tr_first = NNC_TRACE_NOW();
                     tc_fence_after();
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
@@ -272,12 +322,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 if (!ok) break;
                 umma_commit(tfull_bar(acc));
-                if (blockIdx.x == 0) NNC_TRACE_EVENT(202, tr0, tr0, NNC_TRACE_NOW());
+                if (NNC_TRACE_ALL_CTAS || blockIdx.x == 0) NNC_TRACE_EVENT(202, tr0, tr_first, NNC_TRACE_NOW());
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
     } else {  // ---------------- epilogue warps 2..5 ----------------
         const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+        const unsigned long long trk0 = NNC_TRACE_NOW();
+        (void)trk0;
         pdl_wait();
         int acc = 0;
         uint32_t acc_phase = 0;
@@ -298,6 +350,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         if (p.Y_lo) reinterpret_cast<bf16 *>(p.Y_lo)[yo] = __float2bfloat16_rn(a - __bfloat162float(hi));
                     }
                 }
+            } else if (EPI == 2) {
+                // all 32 old values are requested before the first store: a load-add-store chain per token would pay
+                // one memory round trip per token
+                float *y = reinterpret_cast<float *>(p.Y) + m;
+                float old[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) old[i] = (m < p.N && n0 + i < p.T) ? __ldcg(y + (size_t)(n0 + i) * p.ldy) : 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (m < p.N && n0 + i < p.T) y[(size_t)(n0 + i) * p.ldy] = old[i] + __uint_as_float(r[i]);
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -305,35 +367,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     if (m < p.N && t < p.T) {
                         const float v = __uint_as_float(r[i]);
                         if (EPI == 1) reinterpret_cast<bf16 *>(p.Y)[(size_t)t * p.ldy + m] = __float2bfloat16_rn(v);
-                        else if (EPI == 2) reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] += v;
                         else reinterpret_cast<float *>(p.Y)[(size_t)t * p.ldy + m] = v;
                     }
                 }
             }
         };
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            NNC_UNIT_DECODE(tile)
-            (void)kb_lo; (void)kb_hi;
-            const bool got = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4);
-            if (!got && !(SWAP && p.ksplit > 1)) break;
+        WorkIter it(total_tiles, kb_count, stream);
+        Segment g;
+        bool dead = false;   // this warp has seen the abort; in stream mode it keeps walking (the group barriers below
+                             // need all four warps) but touches nothing any more
+        while (it.next(g)) {
+            const int tile_id = g.tile_id;
+            const int mt = tile_id % p.m_tiles, nt = tile_id / p.m_tiles;
+            const bool shared_tile = SWAP && g.n_pieces > 1;
+            const bool got = !dead && mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4);
+            if (!got) {
+                dead = true;
+                if (!stream) break;
+                if (!shared_tile) continue;
+            }
             tc_fence_after();
             const int m = mt * kBM + quarter * 32 + lane;  // D row held by this thread
             const unsigned long long tr0 = NNC_TRACE_NOW();
             unsigned long long tr1 = tr0;
             (void)tr0; (void)tr1;
-            if (SWAP && p.ksplit > 1) {
-                // ---- split K: park this piece's fp32 tile, take a ticket; the piece that arrives last adds the
-                //      pieces in piece order and runs the epilogue (nobody waits) ----
+            if (shared_tile) {
+                // ---- the tile's K range is shared with other CTAs: park this piece's fp32 tile, take a ticket; the
+                //      piece that arrives last adds the pieces in K order and runs the epilogue (nobody waits) ----
                 const int row = quarter * 32 + lane;
-                float *slot = p.part + ((size_t)tile_id * p.ksplit + ks_id) * (size_t)(BN * kBM);
+                constexpr size_t kSlotFloats = (size_t)BN * kBM;
+                float *slot = p.part + (size_t)it.slot_of(blockIdx.x, tile_id) * kSlotFloats;
                 if (got) {
 #pragma unroll 1
                     for (int c0 = 0; c0 < BN; c0 += 32) {
                         uint32_t r[32];
                         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-                        uint4 *dst = reinterpret_cast<uint4 *>(slot + ((size_t)(c0 >> 5) * kBM + row) * 32);
+                        // slot layout [32-column chunk][4-column group][row][4]: a warp's store covers 512 contiguous bytes
+                        uint4 *dst = reinterpret_cast<uint4 *>(slot) + (size_t)(c0 >> 5) * 8 * kBM + row;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                        for (int i = 0; i < 8; ++i) dst[i * kBM] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
                     }
                     tc_fence_before();
                     __syncwarp();
@@ -342,37 +414,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tr1 = NNC_TRACE_NOW();
                 __threadfence();
                 asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (*abort_flag) break;
                 if (warp == 2 && lane == 0) {
-                    const unsigned tk = atomicAdd(&p.tickets[tile_id], 1u);
-                    split_last = (tk == (unsigned)p.ksplit - 1);
-                    if (split_last) p.tickets[tile_id] = 0u;
+                    bool last = false;
+                    if (!*abort_flag) {
+                        const unsigned tk = atomicAdd(&p.tickets[tile_id], 1u);
+                        last = (tk == (unsigned)g.n_pieces - 1);
+                        if (last) p.tickets[tile_id] = 0u;
+                    }
+                    split_last = last;
                 }
                 asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (split_last) {
                     __threadfence();
-                    const float *base = p.part + (size_t)tile_id * p.ksplit * (size_t)(BN * kBM);
 #pragma unroll 1
                     for (int c0 = 0; c0 < BN; c0 += 32) {
                         float sum[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) sum[i] = 0.f;
-                        // pieces are added in piece order; two pieces' loads are in flight at a time
-                        for (int ks = 0; ks < p.ksplit; ks += 2) {
-                            const float4 *s0 = reinterpret_cast<const float4 *>(base + (size_t)ks * (BN * kBM) + ((size_t)(c0 >> 5) * kBM + row) * 32);
-                            const bool two = ks + 1 < p.ksplit;
-                            const float4 *s1 = two ? s0 + (BN * kBM) / 4 : s0;
-                            float4 v0[8], v1[8];
+                        // pieces are added in K order; up to four pieces' loads are in flight at a time
+                        const size_t in_slot = ((size_t)(c0 >> 5) * 8 * kBM + row) * 4;
+                        for (int q0 = 0; q0 < g.n_pieces; q0 += 4) {
+                            float4 v[4][8];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) { v0[i] = __ldcg(s0 + i); v1[i] = __ldcg(s1 + i); }
+                            for (int u = 0; u < 4; ++u) {
+                                if (q0 + u < g.n_pieces) {
+                                    const float4 *src = reinterpret_cast<const float4 *>(
+                                        p.part + (size_t)it.slot_of(g.first_cta + q0 + u, tile_id) * kSlotFloats + in_slot);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                sum[4 * i] += v0[i].x; sum[4 * i + 1] += v0[i].y; sum[4 * i + 2] += v0[i].z; sum[4 * i + 3] += v0[i].w;
+                                    for (int i = 0; i < 8; ++i) v[u][i] = __ldcg(src + i * kBM);
+                                }
                             }
-                            if (two) {
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    sum[4 * i] += v1[i].x; sum[4 * i + 1] += v1[i].y; sum[4 * i + 2] += v1[i].z; sum[4 * i + 3] += v1[i].w;
+                            for (int u = 0; u < 4; ++u) {
+                                if (q0 + u < g.n_pieces) {
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) {
+                                        sum[4 * i] += v[u][i].x; sum[4 * i + 1] += v[u][i].y;
+                                        sum[4 * i + 2] += v[u][i].z; sum[4 * i + 3] += v[u][i].w;
+                                    }
                                 }
                             }
                         }
@@ -382,8 +461,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         store_swap(r, m, nt * BN + c0);
                     }
                 }
-                asm volatile("bar.sync 2, 128;" ::: "memory");   // split_last is rewritten by the next unit
-                if (blockIdx.x == 0 && warp == 2 && lane == 0) NNC_TRACE_EVENT(203, tr0, tr1, NNC_TRACE_NOW());
+                if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0)
+                    NNC_TRACE_EVENT(split_last ? 205 : 203, tr0, tr1, NNC_TRACE_NOW());
+                asm volatile("bar.sync 2, 128;" ::: "memory");   // split_last is rewritten by the next shared tile
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 continue;
             }
@@ -467,6 +547,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (warp == 2 && lane == 0) NNC_TRACE_EVENT(204, trk0, trk0, NNC_TRACE_NOW());
     }
 
     // ---- teardown ----
@@ -540,24 +621,22 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
         p.m_tiles = (N + kBM - 1) / kBM;
         p.n_tiles = (T + BN - 1) / BN;
     }
-    // Few tokens: the product is bound by streaming the weights, and N / 128 output tiles are too few to keep every
-    // SM's loads in flight.  Cut K into pieces so that (tiles x pieces) fills the SMs in whole rounds.
-    p.ksplit = 1; p.part = nullptr; p.tickets = nullptr;
+    // Few tokens: the product is bound by streaming the weights.  Whole tiles dealt round-robin leave SMs idle in the
+    // last round (or all the time, when there are fewer tiles than SMs), so the (tile, K stage) space is cut into one
+    // equal contiguous range per CTA instead; tiles that straddle a cut are finished through partial tiles in scratch.
+    p.stream = 0; p.part = nullptr; p.tickets = nullptr;
+    const int tiles = p.m_tiles * p.n_tiles;
+    int grid = tiles < lc.sm_count ? tiles : lc.sm_count;
     if (SWAP && scratch && scratch->part && scratch->tickets) {
-        const int tiles = p.m_tiles * p.n_tiles, kb_count = K / (kBK * KA);
-        const size_t slot_bytes = (size_t)BN * kBM * 4;
-        double best = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
-        for (int ks = 2; ks <= 16 && best < 0.95; ++ks) {
-            if (kb_count / ks < 2) break;
-            if ((size_t)tiles * ks * slot_bytes > scratch->part_bytes || tiles > scratch->n_tickets) break;
-            const int units = tiles * ks;
-            const double eff = (double)units / (((units + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
-            if (eff > best + 0.02) { best = eff; p.ksplit = ks; }
+        const long long stages = (long long)tiles * (K / (kBK * KA));
+        const int g = stages < lc.sm_count ? (int)stages : lc.sm_count;
+        const double whole_tile_eff = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
+        const size_t need = (size_t)2 * g * BN * kBM * sizeof(float);
+        if (whole_tile_eff < 0.97 && need <= scratch->part_bytes && tiles <= scratch->n_tickets) {
+            p.stream = 1; p.part = scratch->part; p.tickets = scratch->tickets;
+            grid = g;
         }
-        if (p.ksplit > 1) { p.part = scratch->part; p.tickets = scratch->tickets; }
     }
-    int grid = p.m_tiles * p.n_tiles * p.ksplit;
-    if (grid > lc.sm_count) grid = lc.sm_count;
     if (lc.launches) ++*lc.launches;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
