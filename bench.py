@@ -361,6 +361,36 @@ def kernel_roofline_gemm(shape, peaks, T):
             "single_term": {"achieved": round(fl1 / (us1 * 1e-6) / 1e12, 1), "us_per_launch": round(us1, 1)}}
 
 
+def kernel_roofline_attn(shape, peaks, batch, ctx):
+    """The dominant kernel of batched decode at long context -- the split-range flash-decode -- timed alone on a
+    cache of the workload's size (larger than L2); algorithmic bytes = the K and V rows it has to read once."""
+    from paper_2512_21571_b200 import binding
+    nq, nkv = shape.n_q_heads, shape.n_kv_heads
+    max_seq = ctx + 64
+    kc = synth.normal(9, 11, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    vc = synth.normal(9, 12, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    q = synth.normal(9, 13, (batch, nq, 128), 1.0, torch.float32, "cuda")
+    scratch = torch.empty(binding.lib.nnc_attn_scratch_bytes(batch, nq, ctx), dtype=torch.uint8, device="cuda")
+    scratch.zero_()
+    for _ in range(3):
+        binding.op_attn_decode(q, kc, vc, ctx, scratch)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 10
+    e0.record()
+    for _ in range(n):
+        binding.op_attn_decode(q, kc, vc, ctx, scratch)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    nbytes = 2.0 * batch * nkv * ctx * 128 * 2
+    ach = nbytes / (us * 1e-6) / 1e9
+    return {"bound": "hbm", "kernel": "attn_decode_kernel<G=%d>" % (nq // nkv), "shape": [batch, nkv, ctx, 128],
+            "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
+            "peak_source": peaks["source"], "bytes_per_launch": int(nbytes), "us_per_launch": round(us, 2),
+            "launches_timed": n, "traffic": None}
+
+
 # ---- the CPU oracle leg (reported baseline; the only place the product's bench touches oracle/) ------------
 
 def oracle_leg(wl, shape, w_gpu, steps, warmup, budget_s=25.0):
@@ -495,6 +525,8 @@ def main():
         shape = synth.SHAPES[wl["shape"]]
         if wl["kind"] == "decode" and wl["batch"] == 1:
             roof = kernel_roofline_gemv(shape, peaks, None)
+        elif wl["kind"] == "decode":
+            roof = kernel_roofline_attn(shape, peaks, wl["batch"], wl["ctx"])
         else:
             roof = kernel_roofline_gemm(shape, peaks, max(wl["batch"] * wl.get("tokens", 1), 32))
         print(json.dumps({"kernel_only": True, "config": config_of(wl), "roofline": roof}), flush=True)
@@ -540,6 +572,8 @@ def main():
     if rank == 0 and not args.no_extras:
         if wl["kind"] == "decode" and wl["batch"] == 1:
             line["roofline"] = kernel_roofline_gemv(shape, peaks, w)
+        elif wl["kind"] == "decode":
+            line["roofline"] = kernel_roofline_attn(shape, peaks, wl["batch"], wl["ctx"])
         else:
             T = wl["batch"] * wl.get("tokens", 1)
             line["roofline"] = kernel_roofline_gemm(shape, peaks, max(T, 32))

@@ -170,11 +170,14 @@ int nnc_op_gemm(const void *X, const void *X_lo, const void *W, void *Y, int32_t
  * Y bf16 [T][n_out/2], Y[t][i] = silu(gate) * up; n_out a multiple of 16 (rows of Y stay 16-byte aligned). */
 int nnc_op_gemm_swiglu(const void *X, const void *X_lo, const void *W, void *Y, void *Y_lo, int32_t T,
                        int32_t n_out, int32_t n_in, void *cuda_stream); /* Y_lo: NULL or the residual of Y */
-/* nnc_op_gemm for few tokens (T <= 128), where the product is bound by streaming W: K is additionally cut into
- * pieces so that every SM streams a share of W; the fp32 partial tiles meet in `scratch` and the piece that
- * arrives last adds them in piece order (deterministic).  scratch: DEVICE, 256-byte aligned, at least 16 KiB +
- * 1 MiB (more lets larger shapes split); its first 16 KiB are arrival counters that must be zero before the first
- * call and are left zero by every call.  With T > 128 it behaves as nnc_op_gemm. */
+/* nnc_op_gemm for few tokens (T <= 128), where the product is bound by streaming W: the (output tile, K block)
+ * space is cut into one equal contiguous range per SM, so every SM streams the same share of W.  A tile whose K
+ * range straddles a cut is finished through fp32 partial tiles in `scratch`: the CTA holding the tile's first K
+ * piece waits (bounded; on expiry the status word is set) for the others and adds the pieces in K order
+ * (deterministic).  scratch: DEVICE, 256-byte aligned, at least 16 KiB + 2 * 64 KiB * (number of SMs) to cover
+ * every T (a smaller one makes large T fall back to whole tiles); its first 16 KiB are flags that must be zero
+ * before the first call and are left zero by every call that ends without error.  Calls that share a scratch
+ * must not overlap on the device.  With T > 128 it behaves as nnc_op_gemm. */
 int nnc_op_gemm_splitk(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
                        int32_t out_f32, int32_t accumulate, void *scratch, size_t scratch_bytes, void *cuda_stream);
 /* Status word of the nnc_op_* tensor-core kernels (0 = no bounded wait ran out); synchronises the device and

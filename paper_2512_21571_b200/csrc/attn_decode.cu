@@ -54,13 +54,23 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(const Attn
 }  // namespace
 
 int attn_decode_splits(int sm_count, int batch, int nkv, int max_ctx) {
-    // enough CTAs for about two per SM, but never ranges shorter than 64 positions
-    int s = (2 * sm_count + batch * nkv - 1) / (batch * nkv);
-    const int by_len = (max_ctx + 63) / 64;
-    if (s > by_len) s = by_len;
-    if (s > kAttnMaxSplits) s = kAttnMaxSplits;
-    if (s < 1) s = 1;
-    return s;
+    // Two CTAs are resident per SM.  Among the split counts that keep ranges at 64 positions or more, take the one
+    // whose CTA count fills whole rounds of those slots best (a last round that is mostly empty costs a full range's
+    // time), with a small charge per split.
+    const int slots = 2 * sm_count, heads = batch * nkv;
+    int s_max = (max_ctx + 63) / 64;
+    if (s_max > kAttnMaxSplits) s_max = kAttnMaxSplits;
+    if (s_max < 1) s_max = 1;
+    int best = 1;
+    double best_score = -1.0;
+    for (int s = 1; s <= s_max; ++s) {
+        const long long ctas = (long long)heads * s;
+        const long long rounds = (ctas + slots - 1) / slots;
+        const double eff = (double)ctas / (double)(rounds * slots);
+        const double score = eff - 0.002 * s;   // every further split adds a partial result to write and to combine
+        if (score > best_score) { best_score = score; best = s; }
+    }
+    return best;
 }
 
 size_t attn_decode_scratch_floats(int batch, int nq, int n_splits) {

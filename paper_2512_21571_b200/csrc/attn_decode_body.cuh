@@ -10,7 +10,8 @@ namespace nnc {
 constexpr int kPartStride = kHeadDim + 4;  // o~[128], m, l, 2 pad words (rows stay 16-byte aligned)
 constexpr int kAttnWarps = 4;
 constexpr int kSingleRange = 128;    // contexts up to this length are handled by one CTA per KV head
-constexpr int kPrefetchAhead = 6;   // blocks of 16 positions, per warp
+constexpr int kPrefetchAhead = 3;   // blocks of 16 positions, per warp: far enough to cover DRAM latency; much further and a
+                                    // batch of long contexts keeps more prefetched lines in flight than L2 holds on to
 
 __device__ __forceinline__ uint4 ldg_cg(const void *p) {
     uint4 v;

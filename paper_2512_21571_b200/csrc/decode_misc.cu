@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(256)
 rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out,
                     bf16 *__restrict__ out_lo, int H, float eps, int first, int step) {
     __shared__ float red[8];
+    pdl_launch_dependents();   // the next kernel may set itself up (and fetch weights) while this one runs
     pdl_wait();
     const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
     uint2 *dst = reinterpret_cast<uint2 *>(out + (size_t)blockIdx.x * H);
@@ -121,7 +122,6 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
             reinterpret_cast<uint2 *>(out_lo + (size_t)blockIdx.x * H)[i] = r;
         }
     }
-    pdl_launch_dependents();
 }
 
 __global__ void copy_f32_kernel(const float *__restrict__ src, float *__restrict__ dst, size_t n) {

@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_step_mega_kernel(const Meg
 #define NNC_PHASE_END(kid)                                                                          \
     {                                                                                               \
         const unsigned long long t_work__ = NNC_TRACE_NOW();                                        \
+        (void)t_work__;                                                                             \
         if (!grid_barrier(p.bars, bar_k++, p.status)) return;                                       \
         const unsigned long long t_rel__ = NNC_TRACE_NOW();                                         \
         if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 77)) NNC_TRACE_EVENT(kid, t_phase, t_work__, t_rel__); \

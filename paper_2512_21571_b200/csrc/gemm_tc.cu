@@ -131,7 +131,7 @@ struct GemmParams {
     int m_tiles, n_tiles;
     int stream;          // 1: the (tile, K stage) space is cut into one contiguous range per CTA (SWAP only)
     float *part;         // stream: fp32 partial tiles [CTA][first / last segment][BN / 32][8][128 rows][4]
-    uint32_t *tickets;   // stream: one arrival counter per output tile, zero at rest
+    uint32_t *tickets;   // stream: one "piece parked" flag per partial-tile slot, zero at rest
     int *status;
 };
 
@@ -145,7 +145,7 @@ struct Segment {
 //   classic: whole tiles, strided over the grid.
 //   stream:  the tile-major list of all (tile, K stage) pairs is cut into gridDim.x equal contiguous ranges, so every
 //            CTA streams the same number of weight bytes whatever the tile count; a tile whose stages fall into
-//            several ranges is finished by whichever of those CTAs gets there last (see the epilogue).
+//            several ranges is finished by the CTA that holds its first K piece (see the epilogue).
 struct WorkIter {
     int kb_count, tiles, stream;
     long long total;   // stream: tiles * kb_count
@@ -217,6 +217,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ bool split_last;
+    __shared__ __align__(16) uint8_t swiglu_stage[(SWAP && EPI == 3) ? 8192 : 16];   // per epilogue warp: two [32][16] bf16 tiles
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
@@ -248,8 +249,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
+            // The weights depend on nothing that runs before this kernel: the first ring-full of weight tiles is
+            // requested before waiting for the preceding kernel, whose output only the activation tiles read.
+            int ahead = 0;   // stages whose weight tiles are already in flight
+            {
+                WorkIter it(total_tiles, kb_count, stream);
+                Segment g;
+                while (ahead < L::kStages && it.next(g)) {
+                    const int mt = g.tile_id % p.m_tiles, nt = g.tile_id / p.m_tiles;
+                    const int w_row = SWAP ? mt * kBM : nt * BN;
+                    for (int kb = g.kb_lo; kb < g.kb_hi && ahead < L::kStages; ++kb, ++ahead) {
+                        mbar_expect_tx(full_bar(ahead), L::kStage);
+#pragma unroll
+                        for (int a = 0; a < KA; ++a)
+                            tma_load_2d(base + ahead * L::kStage + a * L::kAtom, &map_w, full_bar(ahead), (kb * KA + a) * kBK, w_row);
+                    }
+                }
+            }
             pdl_wait();
-            int stage = 0;
+            int stage = 0, n = 0;
             uint32_t phase = 0;
             bool ok = true;
             WorkIter it(total_tiles, kb_count, stream);
@@ -261,15 +279,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int x_row = SWAP ? nt * BN : mt * kBM;
                 const unsigned long long tr0 = NNC_TRACE_NOW();
                 (void)tr0;
-                for (int kb = kb_lo; kb < kb_hi; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(stage), L::kStage);
+                for (int kb = kb_lo; kb < kb_hi; ++kb, ++n) {
+                    const bool fresh = n >= ahead;   // else: first pass over the ring, weights requested above
+                    if (fresh) {
+                        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(stage), L::kStage);
+                    }
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
                     for (int a = 0; a < KA; ++a) {   // KA consecutive slabs: KA * 128 contiguous bytes of every weight row
                         const uint32_t sa = sw + a * L::kAtom;
                         const int kx = (kb * KA + a) * kBK;
-                        tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
+                        if (fresh) tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
                         tma_load_2d(sa + L::kW, &map_x, full_bar(stage), kx, x_row);
                         if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage), kx, x_row);
                     }
@@ -336,18 +357,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // SWAP stores: row m = weight row, columns = tokens n0 .. n0 + 31; a warp stores 32 consecutive weight rows per token
         auto store_swap = [&](const uint32_t (&r)[32], int m, int n0) {
             if (EPI == 3) {
-                // gate in even lanes, up in odd lanes
+                // Gate rows sit in even lanes, up rows in odd lanes.  The two lanes of a pair swap half of their
+                // values so that each computes 16 of the pair's 32 tokens; the results are staged in this warp's
+                // shared-memory tile [token][16 outputs] and leave as two 16-byte stores per token.
+                const int par = lane & 1, col = lane >> 1;
+                bf16 (*st_hi)[16] = reinterpret_cast<bf16 (*)[16]>(swiglu_stage + (size_t)(quarter * 2) * 1024);
+                bf16 (*st_lo)[16] = reinterpret_cast<bf16 (*)[16]>(swiglu_stage + (size_t)(quarter * 2 + 1) * 1024);
+                float a[16];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float mine = __uint_as_float(r[i]);
-                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                    const int t = n0 + i;
-                    if (!(lane & 1) && m + 1 < p.N && t < p.T) {
-                        const float a = silu_mul(mine, other);
-                        const bf16 hi = __float2bfloat16_rn(a);
-                        const size_t yo = (size_t)t * p.ldy + (m >> 1);
-                        reinterpret_cast<bf16 *>(p.Y)[yo] = hi;
-                        if (p.Y_lo) reinterpret_cast<bf16 *>(p.Y_lo)[yo] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                for (int i = 0; i < 16; ++i) {
+                    const float send = __uint_as_float(par ? r[2 * i] : r[2 * i + 1]);
+                    const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                    const float gate = par ? recv : __uint_as_float(r[2 * i]);
+                    const float up = par ? __uint_as_float(r[2 * i + 1]) : recv;
+                    a[i] = silu_mul(gate, up);   // token n0 + 2 i + par
+                }
+                __syncwarp();   // the previous call's readers are done with the tile
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const bf16 hi = __float2bfloat16_rn(a[i]);
+                    st_hi[2 * i + par][col] = hi;
+                    st_lo[2 * i + par][col] = __float2bfloat16_rn(a[i] - __bfloat162float(hi));
+                }
+                __syncwarp();
+                const int t = n0 + lane;                       // this lane stores token t
+                const int m0 = m - lane;                       // first weight row of this warp (even)
+                if (t < p.T) {
+                    const size_t yo = (size_t)t * p.ldy + (m0 >> 1);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (m0 + 16 * h + 15 < p.N) {          // N is a multiple of 16: a chunk of 8 outputs is whole or absent
+                            *reinterpret_cast<uint4 *>(reinterpret_cast<bf16 *>(p.Y) + yo + 8 * h) =
+                                *reinterpret_cast<const uint4 *>(&st_hi[lane][8 * h]);
+                            if (p.Y_lo)
+                                *reinterpret_cast<uint4 *>(reinterpret_cast<bf16 *>(p.Y_lo) + yo + 8 * h) =
+                                    *reinterpret_cast<const uint4 *>(&st_lo[lane][8 * h]);
+                        }
                     }
                 }
             } else if (EPI == 2) {
@@ -392,78 +437,114 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             unsigned long long tr1 = tr0;
             (void)tr0; (void)tr1;
             if (shared_tile) {
-                // ---- the tile's K range is shared with other CTAs: park this piece's fp32 tile, take a ticket; the
-                //      piece that arrives last adds the pieces in K order and runs the epilogue (nobody waits) ----
+                // ---- the tile's K range is shared with other CTAs.  Every piece but the first parks its fp32 tile in
+                //      scratch and raises its flag.  The first piece is the last segment of its CTA's range, so it is
+                //      the one that finishes last by schedule: it keeps its tile in tensor memory, waits (bounded) for
+                //      the other flags, adds the pieces in K order and runs the epilogue. ----
                 const int row = quarter * 32 + lane;
                 constexpr size_t kSlotFloats = (size_t)BN * kBM;
-                float *slot = p.part + (size_t)it.slot_of(blockIdx.x, tile_id) * kSlotFloats;
-                if (got) {
+                if (g.piece != 0) {
+                    const int my_slot = it.slot_of(blockIdx.x, tile_id);
+                    float *slot = p.part + (size_t)my_slot * kSlotFloats;
+                    if (got) {
 #pragma unroll 1
-                    for (int c0 = 0; c0 < BN; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-                        // slot layout [32-column chunk][4-column group][row][4]: a warp's store covers 512 contiguous bytes
-                        uint4 *dst = reinterpret_cast<uint4 *>(slot) + (size_t)(c0 >> 5) * 8 * kBM + row;
+                        for (int c0 = 0; c0 < BN; c0 += 32) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                            // slot layout [32-column chunk][4-column group][row][4]: a warp's store covers 512 contiguous bytes
+                            uint4 *dst = reinterpret_cast<uint4 *>(slot) + (size_t)(c0 >> 5) * 8 * kBM + row;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i * kBM] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                            for (int i = 0; i < 8; ++i) dst[i * kBM] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar(acc));
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(acc));
-                }
-                tr1 = NNC_TRACE_NOW();
-                __threadfence();
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (warp == 2 && lane == 0) {
-                    bool last = false;
-                    if (!*abort_flag) {
-                        const unsigned tk = atomicAdd(&p.tickets[tile_id], 1u);
-                        last = (tk == (unsigned)g.n_pieces - 1);
-                        if (last) p.tickets[tile_id] = 0u;
+                    tr1 = NNC_TRACE_NOW();
+                    asm volatile("bar.sync 2, 128;" ::: "memory");   // all four warps' stores are issued
+                    if (warp == 2 && lane == 0 && !*abort_flag) {
+                        __threadfence();
+                        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + my_slot), "r"(1u) : "memory");
                     }
-                    split_last = last;
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (split_last) {
-                    __threadfence();
-#pragma unroll 1
-                    for (int c0 = 0; c0 < BN; c0 += 32) {
-                        float sum[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) sum[i] = 0.f;
-                        // pieces are added in K order; up to four pieces' loads are in flight at a time
-                        const size_t in_slot = ((size_t)(c0 >> 5) * 8 * kBM + row) * 4;
-                        for (int q0 = 0; q0 < g.n_pieces; q0 += 4) {
-                            float4 v[4][8];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                if (q0 + u < g.n_pieces) {
-                                    const float4 *src = reinterpret_cast<const float4 *>(
-                                        p.part + (size_t)it.slot_of(g.first_cta + q0 + u, tile_id) * kSlotFloats + in_slot);
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i) v[u][i] = __ldcg(src + i * kBM);
-                                }
-                            }
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                if (q0 + u < g.n_pieces) {
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i) {
-                                        sum[4 * i] += v[u][i].x; sum[4 * i + 1] += v[u][i].y;
-                                        sum[4 * i + 2] += v[u][i].z; sum[4 * i + 3] += v[u][i].w;
+                    if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(203, tr0, tr1, NNC_TRACE_NOW());
+                } else {
+                    if (warp == 2 && lane == 0) {
+                        // bounded wait for the other pieces (they never wait for anything of this CTA's)
+                        bool ok = got;
+                        unsigned long long t_first = 0;
+                        for (int q = 1; q < g.n_pieces && ok; ++q) {
+                            const uint32_t *flag = p.tickets + it.slot_of(g.first_cta + q, tile_id);
+                            for (uint32_t spin = 0;; ++spin) {
+                                uint32_t v;
+                                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                                if (v) break;
+                                if ((spin & 255u) == 255u) {
+                                    const unsigned long long now = global_ns();
+                                    if (t_first == 0) t_first = now;
+                                    if (*abort_flag || now - t_first > kWaitLimitNs) {
+                                        if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 5); }
+                                        ok = false;
+                                        break;
                                     }
                                 }
                             }
                         }
-                        uint32_t r[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i]);
-                        store_swap(r, m, nt * BN + c0);
+                        split_last = ok;
                     }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    tr1 = NNC_TRACE_NOW();
+                    if (split_last && got) {
+#pragma unroll 1
+                        for (int c0 = 0; c0 < BN; c0 += 32) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                            float sum[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) sum[i] = __uint_as_float(r[i]);
+                            // the parked pieces are added in K order; up to four pieces' loads are in flight at a time
+                            const size_t in_slot = ((size_t)(c0 >> 5) * 8 * kBM + row) * 4;
+                            for (int q0 = 1; q0 < g.n_pieces; q0 += 4) {
+                                float4 v[4][8];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    if (q0 + u < g.n_pieces) {
+                                        const float4 *src = reinterpret_cast<const float4 *>(
+                                            p.part + (size_t)it.slot_of(g.first_cta + q0 + u, tile_id) * kSlotFloats + in_slot);
+#pragma unroll
+                                        for (int i = 0; i < 8; ++i) v[u][i] = __ldcg(src + i * kBM);
+                                    }
+                                }
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    if (q0 + u < g.n_pieces) {
+#pragma unroll
+                                        for (int i = 0; i < 8; ++i) {
+                                            sum[4 * i] += v[u][i].x; sum[4 * i + 1] += v[u][i].y;
+                                            sum[4 * i + 2] += v[u][i].z; sum[4 * i + 3] += v[u][i].w;
+                                        }
+                                    }
+                                }
+                            }
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i]);
+                            const unsigned long long tr2 = NNC_TRACE_NOW();
+                            (void)tr2;
+                            store_swap(r, m, nt * BN + c0);
+                            if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(206, tr1, tr2, NNC_TRACE_NOW());
+                        }
+                    }
+                    if (got) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar(acc));
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");   // every warp has read the parked pieces
+                    if (warp == 2 && lane == 0 && split_last) {
+                        // flags back to rest for the next launch that uses this scratch
+                        for (int q = 1; q < g.n_pieces; ++q) p.tickets[it.slot_of(g.first_cta + q, tile_id)] = 0u;
+                    }
+                    if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(205, tr0, tr1, NNC_TRACE_NOW());
                 }
-                if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0)
-                    NNC_TRACE_EVENT(split_last ? 205 : 203, tr0, tr1, NNC_TRACE_NOW());
-                asm volatile("bar.sync 2, 128;" ::: "memory");   // split_last is rewritten by the next shared tile
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 continue;
             }
@@ -632,7 +713,7 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
         const int g = stages < lc.sm_count ? (int)stages : lc.sm_count;
         const double whole_tile_eff = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
         const size_t need = (size_t)2 * g * BN * kBM * sizeof(float);
-        if (whole_tile_eff < 0.97 && need <= scratch->part_bytes && tiles <= scratch->n_tickets) {
+        if (whole_tile_eff < 0.97 && need <= scratch->part_bytes && 2 * g <= scratch->n_tickets) {
             p.stream = 1; p.part = scratch->part; p.tickets = scratch->tickets;
             grid = g;
         }
@@ -697,7 +778,7 @@ cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, co
     // the epilogue stores 16-byte vectors per output row: the row pitch must keep them aligned
     const bool out_bf16 = epi == kEpiStoreBf16 || epi == kEpiSwigluBf16;
     if (ldy % (out_bf16 ? 8 : 4) != 0) return cudaErrorInvalidValue;
-    if (epi == kEpiSwigluBf16 && N % 2 != 0) return cudaErrorInvalidValue;
+    if (epi == kEpiSwigluBf16 && N % 16 != 0) return cudaErrorInvalidValue;   // outputs leave in chunks of 8
     return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch)
                 : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch);
 }
