@@ -145,10 +145,14 @@ def test_gemm_split_activations_recover_fp32_inputs(nnc, oracle_mod, T, N, K):
     assert nnc.op_status() == 0
 
 
-@pytest.mark.parametrize("T,N,K", [(32, 4096, 4096), (7, 384, 640), (128, 1024, 2048), (33, 1000, 1024), (32, 4096, 12288)])
+@pytest.mark.parametrize("T,N,K", [(32, 4096, 4096), (7, 384, 640), (128, 1024, 2048), (33, 1000, 1024), (32, 4096, 12288),
+                                   (1, 128, 256), (64, 6144, 4096), (100, 24576, 1024), (32, 151936, 256), (17, 136, 8192)])
 def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
-    """Few tokens: K is cut into pieces across CTAs and the fp32 partial tiles are added in piece order.  Same
-    result as the oracle's matmul, bit-identical from run to run, scratch counters left at zero."""
+    """Few tokens: the (output tile, K stage) list is cut into one contiguous range per CTA; tiles that straddle a
+    cut are finished from fp32 partial tiles added in K order.  Covers a single tile with a single stage (one CTA),
+    fewer tiles than SMs (every tile shared by several CTAs), more tiles than SMs (most tiles whole), ragged N and
+    K that is not a multiple of the 4-slab stage.  Same result as the oracle's matmul, bit-identical from run to
+    run, scratch flags left at zero."""
     X = synth.normal(8, 1, (T, K), 1.0, torch.float32, "cuda")
     W = _w(8, 2, (N, K))
     hi, lo = nnc.split_bf16(X)
