@@ -249,25 +249,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
-            // The weights depend on nothing that runs before this kernel: the first ring-full of weight tiles is
-            // requested before waiting for the preceding kernel, whose output only the activation tiles read.
-            int ahead = 0;   // stages whose weight tiles are already in flight
-            {
-                WorkIter it(total_tiles, kb_count, stream);
-                Segment g;
-                while (ahead < L::kStages && it.next(g)) {
-                    const int mt = g.tile_id % p.m_tiles, nt = g.tile_id / p.m_tiles;
-                    const int w_row = SWAP ? mt * kBM : nt * BN;
-                    for (int kb = g.kb_lo; kb < g.kb_hi && ahead < L::kStages; ++kb, ++ahead) {
-                        mbar_expect_tx(full_bar(ahead), L::kStage);
-#pragma unroll
-                        for (int a = 0; a < KA; ++a)
-                            tma_load_2d(base + ahead * L::kStage + a * L::kAtom, &map_w, full_bar(ahead), (kb * KA + a) * kBK, w_row);
-                    }
-                }
-            }
             pdl_wait();
-            int stage = 0, n = 0;
+            int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             WorkIter it(total_tiles, kb_count, stream);
@@ -279,18 +262,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int x_row = SWAP ? nt * BN : mt * kBM;
                 const unsigned long long tr0 = NNC_TRACE_NOW();
                 (void)tr0;
-                for (int kb = kb_lo; kb < kb_hi; ++kb, ++n) {
-                    const bool fresh = n >= ahead;   // else: first pass over the ring, weights requested above
-                    if (fresh) {
-                        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(stage), L::kStage);
-                    }
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(stage), L::kStage);
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
                     for (int a = 0; a < KA; ++a) {   // KA consecutive slabs: KA * 128 contiguous bytes of every weight row
                         const uint32_t sa = sw + a * L::kAtom;
                         const int kx = (kb * KA + a) * kBK;
-                        if (fresh) tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
+                        tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
                         tma_load_2d(sa + L::kW, &map_x, full_bar(stage), kx, x_row);
                         if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage), kx, x_row);
                     }
