@@ -68,18 +68,22 @@ static void trace_bind_this_tu(TraceRec *buf, unsigned *cnt) {
 }
 namespace { struct TraceRegistrar { TraceRegistrar() { trace_register(&trace_bind_this_tu); } } g_trace_registrar; }
 struct TraceScope {
-    unsigned kid, mark, mark2, mark3; unsigned long long t0;
+    unsigned kid, mark, mark2, mark3, c0; unsigned long long t0;   // c0: SM cycle counter at entry (the record keeps the cycles spent)
     __device__ __forceinline__ unsigned since() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (unsigned)(t - t0); }
     __device__ __forceinline__ void set_mark() { mark = since(); }
     __device__ __forceinline__ void set_mark2() { mark2 = since(); }
     __device__ __forceinline__ void set_mark3() { mark3 = since(); }
-    __device__ __forceinline__ TraceScope(unsigned k) : kid(k), mark(0), mark2(0), mark3(0) { asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0)); }
+    __device__ __forceinline__ TraceScope(unsigned k) : kid(k), mark(0), mark2(0), mark3(0) {
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+        asm volatile("mov.u32 %0, %clock;" : "=r"(c0));
+    }
     __device__ __forceinline__ ~TraceScope() {
         if (threadIdx.x == 0 && g_trace_buf) {
             unsigned long long t1; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
             unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+            unsigned c1; asm volatile("mov.u32 %0, %clock;" : "=r"(c1));
             const unsigned i = atomicAdd(g_trace_cnt, 1u);
-            if (i < kTraceMax) g_trace_buf[i] = TraceRec{kid, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), sm, mark, t0, t1, mark2, mark3, 0, 0};
+            if (i < kTraceMax) g_trace_buf[i] = TraceRec{kid, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), sm, mark, t0, t1, mark2, mark3, c1 - c0, 0};
         }
     }
 };
