@@ -361,6 +361,11 @@ def kernel_roofline_gemm(shape, peaks, T):
             "single_term": {"achieved": round(fl1 / (us1 * 1e-6) / 1e12, 1), "us_per_launch": round(us1, 1)}}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the flash-decode from one ncu capture of this very
+# configuration (profiles/attn_decode_kernel_qwen3-8b_b32_ctx8192.md); to be set back to None when the kernel changes
+ATTN_DRAM_TRAFFIC = {(32, 8, 32, 8192): 1.0831e9}
+
+
 def kernel_roofline_attn(shape, peaks, batch, ctx):
     """The dominant kernel of batched decode at long context -- the split-range flash-decode -- timed alone on a
     cache of the workload's size (larger than L2); algorithmic bytes = the K and V rows it has to read once."""
@@ -388,7 +393,7 @@ def kernel_roofline_attn(shape, peaks, batch, ctx):
     return {"bound": "hbm", "kernel": "attn_decode_kernel<G=%d>" % (nq // nkv), "shape": [batch, nkv, ctx, 128],
             "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
             "peak_source": peaks["source"], "bytes_per_launch": int(nbytes), "us_per_launch": round(us, 2),
-            "launches_timed": n, "traffic": None}
+            "launches_timed": n, "traffic": ATTN_DRAM_TRAFFIC.get((nq, nkv, batch, ctx))}
 
 
 # ---- the CPU oracle leg (reported baseline; the only place the product's bench touches oracle/) ------------
