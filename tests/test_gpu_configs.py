@@ -3,7 +3,7 @@ oracle's tokens.  Weights are generated once on the GPU (seeded) and copied to t
 
 Sizes the oracle cannot finish in reasonable time are sampled: the number of oracle decode steps is bounded
 (NNC_TEST_STEPS overrides), and batched workloads are checked on a subset of sequences plus the
-batch-independence property.  Error statistics are appended to gpurun_out/parity_stats.txt.
+batch-independence property.  Error statistics are printed and, if NNC_PARITY_STATS names a file, appended to it.
 """
 import os
 import time
@@ -21,9 +21,11 @@ STEPS = int(os.environ.get("NNC_TEST_STEPS", "0"))
 
 
 def _log(line):
-    os.makedirs("gpurun_out", exist_ok=True)
-    with open("gpurun_out/parity_stats.txt", "a") as f:
-        f.write(line + "\n")
+    path = os.environ.get("NNC_PARITY_STATS")
+    if path:
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        with open(path, "a") as f:
+            f.write(line + "\n")
     print(line)
 
 
