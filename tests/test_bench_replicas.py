@@ -21,7 +21,7 @@ _RANK_PROGRAM = textwrap.dedent("""
     assert bench.max_over_ranks(7.0 - rank, world) == 7.0
     dist.barrier()
     dist.destroy_process_group()
-    sys.stdout.write("rank %d ok\n" % rank)   # one write per rank: the two ranks share the pipe
+    sys.stdout.write("rank %d ok\\n" % rank)   # one write per rank: the two ranks share the pipe
     sys.stdout.flush()
 """)
 
