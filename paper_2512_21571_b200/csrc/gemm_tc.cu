@@ -448,28 +448,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(203, tr0, tr1, NNC_TRACE_NOW());
                 } else {
-                    if (warp == 2 && lane == 0) {
-                        // bounded wait for the other pieces (they never wait for anything of this CTA's)
+                    if (warp == 2) {
+                        // bounded wait for the other pieces (they never wait for anything of this CTA's); one flag per
+                        // lane, so that all of them are polled in one memory round trip
                         bool ok = got;
                         unsigned long long t_first = 0;
-                        for (int q = 1; q < g.n_pieces && ok; ++q) {
-                            const uint32_t *flag = p.tickets + it.slot_of(g.first_cta + q, tile_id);
+                        for (int q0 = 1; q0 < g.n_pieces && ok; q0 += 32) {
+                            const int q = q0 + lane;
+                            const uint32_t *flag = (q < g.n_pieces) ? p.tickets + it.slot_of(g.first_cta + q, tile_id) : nullptr;
                             for (uint32_t spin = 0;; ++spin) {
-                                uint32_t v;
-                                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-                                if (v) break;
+                                uint32_t v = 1u;
+                                if (flag) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                                if (__all_sync(0xffffffffu, v != 0u)) break;
                                 if ((spin & 255u) == 255u) {
-                                    const unsigned long long now = global_ns();
-                                    if (t_first == 0) t_first = now;
-                                    if (*abort_flag || now - t_first > kWaitLimitNs) {
-                                        if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 5); }
-                                        ok = false;
-                                        break;
+                                    int give_up = 0;
+                                    if (lane == 0) {
+                                        const unsigned long long now = global_ns();
+                                        if (t_first == 0) t_first = now;
+                                        if (*abort_flag || now - t_first > kWaitLimitNs) {
+                                            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 5); }
+                                            give_up = 1;
+                                        }
                                     }
+                                    if (__shfl_sync(0xffffffffu, give_up, 0)) { ok = false; break; }
                                 }
                             }
                         }
-                        split_last = ok;
+                        if (lane == 0) split_last = ok;
                     }
                     asm volatile("bar.sync 2, 128;" ::: "memory");
                     tr1 = NNC_TRACE_NOW();
