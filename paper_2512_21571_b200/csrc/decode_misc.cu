@@ -90,12 +90,24 @@ __global__ void __launch_bounds__(256)
 rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out,
                     bf16 *__restrict__ out_lo, int H, float eps, int first, int step) {
     __shared__ float red[8];
-    pdl_launch_dependents();   // the next kernel may set itself up (and fetch weights) while this one runs
+    pdl_launch_dependents();   // the next kernel may set itself up while this one runs
     pdl_wait();
     const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
     uint2 *dst = reinterpret_cast<uint2 *>(out + (size_t)blockIdx.x * H);
+    // rows of up to 4096 elements stay in registers between the two passes (4 x 16 bytes per thread, all requested
+    // at once); longer rows are read again
+    constexpr int kKeep = 4;
+    const int n4 = H / 4;
+    float4 keep[kKeep];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < H / 4; i += 256) {
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const int i = threadIdx.x + 256 * u;
+        keep[u] = (i < n4) ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) ss += keep[u].x * keep[u].x + keep[u].y * keep[u].y + keep[u].z * keep[u].z + keep[u].w * keep[u].w;
+    for (int i = threadIdx.x + 256 * kKeep; i < n4; i += 256) {
         const float4 v = src[i];
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
@@ -106,8 +118,7 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)H + eps);
-    for (int i = threadIdx.x; i < H / 4; i += 256) {
-        const float4 v = src[i];
+    auto emit = [&](int i, const float4 &v) {
         const uint2 g = reinterpret_cast<const uint2 *>(gain)[i];
         const float y0 = v.x * inv * bf16_lo(g.x), y1 = v.y * inv * bf16_hi(g.x);
         const float y2 = v.z * inv * bf16_lo(g.y), y3 = v.w * inv * bf16_hi(g.y);
@@ -121,7 +132,13 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
             r.y = pack_bf16x2(y2 - bf16_lo(o.y), y3 - bf16_hi(o.y));
             reinterpret_cast<uint2 *>(out_lo + (size_t)blockIdx.x * H)[i] = r;
         }
+    };
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const int i = threadIdx.x + 256 * u;
+        if (i < n4) emit(i, keep[u]);
     }
+    for (int i = threadIdx.x + 256 * kKeep; i < n4; i += 256) emit(i, src[i]);
 }
 
 __global__ void copy_f32_kernel(const float *__restrict__ src, float *__restrict__ dst, size_t n) {
