@@ -75,6 +75,12 @@ def load(double_acc: bool = False) -> C.CDLL:
         L.orc_softmax.argtypes = [C.c_void_p, C.c_int]
         L.orc_attend.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_size_t,
                                  C.c_void_p, C.c_void_p]
+        L.orc_e4m3_to_f32.restype = C.c_float
+        L.orc_e4m3_to_f32.argtypes = [C.c_uint8]
+        L.orc_f32_to_e4m3.restype = C.c_uint8
+        L.orc_f32_to_e4m3.argtypes = [C.c_float]
+        L.orc_quantise_rows_e4m3.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_dequantise_rows_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         L.orc_argmax_margin.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         _LIBS[double_acc] = L
     return _LIBS[double_acc]
@@ -140,7 +146,35 @@ def attend(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, double_acc=False) 
 def argmax_margin(v: torch.Tensor):
     idx, margin = C.c_int32(), C.c_float()
     load().orc_argmax_margin(_f32(v).data_ptr(), v.numel(), C.byref(idx), C.byref(margin))
+    if idx.value < 0:
+        raise ValueError("argmax_margin: the logits hold a NaN or an infinity")
     return idx.value, margin.value
+
+
+def e4m3_to_f32(code: int) -> float:
+    return load().orc_e4m3_to_f32(code)
+
+
+def f32_to_e4m3(x: float) -> int:
+    return load().orc_f32_to_e4m3(x)
+
+
+def quantise_rows_e4m3(W: torch.Tensor):
+    """bf16 [n_out][n_in] -> (codes uint8 [n_out][n_in], exps int8 [n_out]): E4M3 codes of W / 2^exp per row."""
+    n_out, n_in = W.shape
+    codes = torch.empty(n_out, n_in, dtype=torch.uint8)
+    exps = torch.empty(n_out, dtype=torch.int8)
+    load().orc_quantise_rows_e4m3(_bf16(W).data_ptr(), n_out, n_in, codes.data_ptr(), exps.data_ptr())
+    return codes, exps
+
+
+def dequantise_rows_e4m3(codes: torch.Tensor, exps: torch.Tensor) -> torch.Tensor:
+    """(codes, exps) -> bf16 [n_out][n_in] holding e4m3(code) * 2^exp exactly."""
+    n_out, n_in = codes.shape
+    assert codes.dtype == torch.uint8 and exps.dtype == torch.int8 and codes.is_contiguous() and exps.is_contiguous()
+    W = torch.empty(n_out, n_in, dtype=torch.bfloat16)
+    load().orc_dequantise_rows_e4m3(codes.data_ptr(), exps.data_ptr(), n_out, n_in, W.data_ptr())
+    return W
 
 
 def f32_to_bf16_bits(f: float) -> int:

@@ -107,6 +107,73 @@ void orc_matmul(const uint16_t *W, const float *X, int T, int n_out, int n_in, f
             Y[(size_t)t * n_out + o] = dot_bf16_f32(W + (size_t)o * n_in, X + (size_t)t * n_in, n_in);
 }
 
+/* ------------------------------------------------------ second weight precision: FP8 E4M3, row scales */
+/* The paper evaluates two weight precisions of the same models (Section 4.1: F32 and F16 variants).  The second
+ * precision of this build is weight-only FP8: every weight row is stored as E4M3 codes (1 sign, 4 exponent bits
+ * with bias 7, 3 mantissa bits; exponent 0 = subnormal m * 2^-9; no infinities, S.1111.111 = NaN, largest finite
+ * value 448) times one power-of-two scale 2^e per output row.  Reading taken (the paper is silent on quantisation):
+ *   e     = the smallest integer with max_k |W[o][k]| <= 448 * 2^e  (0 for an all-zero row),
+ *   code  = round-to-nearest-even of W[o][k] / 2^e onto the E4M3 grid, saturating at +-448,
+ *   value = e4m3(code) * 2^e -- at most 4 significant bits times a power of two, hence exactly a bf16 value.
+ * A model "in FP8" is the same forward pass on the dequantised bf16 matrices, so every other function of this
+ * file applies unchanged. */
+float orc_e4m3_to_f32(uint8_t c) {
+    const int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    float v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexpf((float)m, -9);
+    else v = ldexpf(1.0f + (float)m / 8.0f, e - 7);
+    return sign ? -v : v;
+}
+
+uint8_t orc_f32_to_e4m3(float x) {
+    const uint8_t sign = signbit(x) ? 0x80 : 0;
+    const float a = fabsf(x);
+    if (isnan(x)) return 0x7f;
+    if (a > 448.0f) return sign | 0x7e;                       /* saturate: 0x7e is 448 */
+    if (a < 0.015625f) {                                      /* below 2^-6: the subnormal grid, step 2^-9 */
+        const int q = (int)rintf(ldexpf(a, 9));               /* exact scaling; rintf rounds to nearest even */
+        return sign | (uint8_t)q;                             /* q == 8 is the smallest normal, code 0x08 */
+    }
+    int E;
+    const float f = frexpf(a, &E);                            /* a = f * 2^E, f in [0.5, 1) */
+    int q = (int)rintf((2.0f * f - 1.0f) * 8.0f);             /* mantissa steps of 1/8 above 2^(E-1) */
+    int e = E - 1 + 7;
+    if (q == 8) { q = 0; ++e; }
+    return sign | (uint8_t)((e << 3) | q);                    /* a <= 448 keeps this at or below 0x7e */
+}
+
+/* W bf16 [n_out][n_in] -> codes [n_out][n_in], exps [n_out] */
+void orc_quantise_rows_e4m3(const uint16_t *W, int n_out, int n_in, uint8_t *codes, int8_t *exps) {
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < n_out; ++o) {
+        const uint16_t *row = W + (size_t)o * n_in;
+        float amax = 0.0f;
+        for (int k = 0; k < n_in; ++k) {
+            const float a = fabsf(orc_bf16_to_f32(row[k]));
+            if (a > amax) amax = a;
+        }
+        int e = 0;
+        if (amax > 0.0f) {
+            int E;
+            const float f = frexpf(amax, &E);                 /* 448 = 0.875 * 2^9 */
+            e = (f <= 0.875f) ? E - 9 : E - 8;
+            if (e < -127) e = -127;
+            if (e > 127) e = 127;
+        }
+        exps[o] = (int8_t)e;
+        for (int k = 0; k < n_in; ++k)
+            codes[(size_t)o * n_in + k] = orc_f32_to_e4m3(ldexpf(orc_bf16_to_f32(row[k]), -e));
+    }
+}
+
+void orc_dequantise_rows_e4m3(const uint8_t *codes, const int8_t *exps, int n_out, int n_in, uint16_t *W) {
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < n_out; ++o)
+        for (int k = 0; k < n_in; ++k)
+            W[(size_t)o * n_in + k] = orc_f32_to_bf16(ldexpf(orc_e4m3_to_f32(codes[(size_t)o * n_in + k]), exps[o]));
+}
+
 /* ------------------------------------------------------------------------------------- softmax / SwiGLU */
 float orc_silu(float z) { return (float)((acc_t)z / ((acc_t)1 + ORC_EXP(-(acc_t)z))); }
 
@@ -142,8 +209,15 @@ void orc_attend(const float *q, const uint16_t *K, const uint16_t *V, int n, int
     }
 }
 
-/* argmax with lowest index on ties, and the gap between the two largest values */
+/* argmax with lowest index on ties, and the gap between the two largest values.  Logits must be finite: a NaN
+ * or an infinity anywhere is reported as index -1 with a NaN margin, never silently ranked. */
 void orc_argmax_margin(const float *v, int n, int32_t *idx, float *margin) {
+    for (int i = 0; i < n; ++i)
+        if (!isfinite(v[i])) {
+            *idx = -1;
+            *margin = NAN;
+            return;
+        }
     int best = 0;
     for (int i = 1; i < n; ++i)
         if (v[i] > v[best]) best = i;

@@ -143,6 +143,10 @@ def test_silu_and_argmax(oracle_mod):
     assert idx == 1 and margin == 0.0
     idx, margin = oracle_mod.argmax_margin(torch.tensor([0.5, 2.0, -1.0, 2.25, 1.5]))
     assert idx == 3 and margin == 0.25
+    # non-finite logits are an error, never a rank
+    for bad in (float("nan"), float("inf"), float("-inf")):
+        with pytest.raises(ValueError):
+            oracle_mod.argmax_margin(torch.tensor([0.5, bad, 1.0]))
 
 
 # ----------------------------------------------------------------------------------------------- matmul
