@@ -61,6 +61,9 @@ typedef struct {
                              * mantissa bits, which keeps deep models inside the parity tolerance at twice the
                              * tensor-core work.  1: one bf16 term (half the tensor-core work; rounding error of
                              * 2^-9 per operand accumulates to a few percent over ~30 layers). */
+    int32_t serial_launches; /* 0 (default): kernels are launched with programmatic stream serialization, so a
+                             * kernel's set-up and weight prefetch overlap its predecessor's tail.  1: plain stream
+                             * order (for debugging and for timing the overlap's worth). */
 } nnc_config;
 
 /* Per-layer weights: DEVICE pointers, bf16.  Read only during nnc_model_create (they are repacked into the

@@ -24,7 +24,8 @@ lib = C.CDLL(LIB_PATH)
 class nnc_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "intermediate",
                                          "vocab", "max_seq", "max_batch", "max_tokens", "tie_embeddings")] + \
-               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("fast_bf16_activations", C.c_int32)]
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("fast_bf16_activations", C.c_int32),
+                ("serial_launches", C.c_int32)]
 
 
 LAYER_FIELDS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "g_in", "g_post", "g_q", "g_k")
@@ -100,13 +101,13 @@ class Model:
     """nnc_model_create / nnc_prefill / nnc_decode_step and the auxiliary calls, one method per C function."""
 
     def __init__(self, shape, weights: dict, max_seq: int, max_batch: int = 1, max_tokens: Optional[int] = None,
-                 fast_bf16_activations: bool = False):
+                 fast_bf16_activations: bool = False, serial_launches: bool = False):
         self.shape = shape
         self.cfg = nnc_config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                               shape.intermediate, shape.vocab, max_seq, max_batch,
                               max_tokens if max_tokens is not None else max(max_batch, 1),
                               int(shape.tie_embeddings), shape.rms_eps, shape.rope_theta,
-                              int(fast_bf16_activations))
+                              int(fast_bf16_activations), int(serial_launches))
         self.handle = C.c_void_p()
         nbytes = lib.nnc_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
@@ -222,12 +223,6 @@ class Model:
 def _ok(rc: int, what: str):
     if rc:
         raise NncError(rc, what)
-
-
-def split_bf16(x: torch.Tensor):
-    """fp32 -> (hi, lo) bf16 pair with hi + lo ~ x to 16 mantissa bits (input marshalling for op_gemm)."""
-    hi = x.to(torch.bfloat16)
-    return hi, (x - hi.float()).to(torch.bfloat16)
 
 
 def op_gemm(X: torch.Tensor, W: torch.Tensor, out_f32: bool = True, accumulate_into: Optional[torch.Tensor] = None,

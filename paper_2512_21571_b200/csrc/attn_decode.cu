@@ -5,11 +5,13 @@
 // wide loads and few instructions per byte:
 //   - grid (n_splits, n_kv_heads, batch), 4 warps.  A CTA owns one KV head and one contiguous range of
 //     positions; its G query heads ride along, so every K/V byte is loaded once and feeds G dot products.
-//   - the two products run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 accumulate) with
-//     the G query heads as the (padded) 16-row operand.  Q and the probabilities are fed as two bf16 terms each
-//     (value + rounding residual), so the result keeps fp32-level accuracy.  K and V fragments are loaded
-//     straight from global memory as 16-byte vectors: the contraction index of Q.K^T (the head dimension) and the
-//     output column index of P.V are permuted so that what a thread needs is contiguous in the cache row.
+//   - the two products run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 accumulate) in
+//     transposed form: S^T = K Q^T and O^T = V^T P^T, so 16 cached positions (resp. 16 head-dimension elements)
+//     fill the 16-row operand and the G <= 8 query heads are the 8-column operand -- no padding rows.  Q and the
+//     probabilities are fed as two bf16 terms each (value + rounding residual), so the result keeps fp32-level
+//     accuracy.  K and V fragments are loaded straight from global memory as 16-byte vectors: the contraction
+//     index of K Q^T (the head dimension) and the row index of V^T P^T are permuted so that what a thread needs
+//     is contiguous in the cache row.
 //   - every warp walks its own blocks of 16 positions with a private online softmax; warps, then CTAs, are
 //     merged through (m, l, o~) partials.  The CTA that finishes last for a (sequence, KV head) folds the
 //     partials in split order (a ticket counter; nobody waits), so the result does not depend on arrival order.

@@ -1,6 +1,6 @@
 // Body of the GQA split-K flash-decode (see attn_decode.cu for the design): one 4-warp group handles one
-// (sequence, KV head, position range).  Shared by the stand-alone kernel and the whole-step decode kernel, which
-// runs two such groups per CTA; the group synchronises on its own named barrier.
+// (sequence, KV head, position range) and synchronises on a named barrier of its own, so the body can be placed
+// in kernels that hold other warps besides the group.
 #pragma once
 #include "common.cuh"
 #include "nnc_internal.h"

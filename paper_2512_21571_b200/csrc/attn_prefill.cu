@@ -105,7 +105,8 @@ attn_prefill_kernel(const float *__restrict__ qkv, int rows_per_seq, const bf16 
         }
     }
 
-    const int n_keys = min(P0 + q0 + kBM, P0 + T);       // cache positions the last row of this tile may see
+    // cache positions the last row of this tile may see; never past the head's slab, whatever the caller put in *d_len
+    const int n_keys = min(min(P0 + q0 + kBM, P0 + T), max_seq);
     const int n_tiles = (n_keys + kBN - 1) / kBN;
     const size_t head_off = ((size_t)seq * nkv + j) * (size_t)max_seq * kHeadDim;
     const bf16 *kbase = kcache + head_off, *vbase = vcache + head_off;
@@ -230,13 +231,9 @@ attn_prefill_kernel(const float *__restrict__ qkv, int rows_per_seq, const bf16 
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
                                 const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
                                 const int32_t *d_len) {
-    static bool attr_done = false;
+    static unsigned long long attr_done = 0;   // one bit per device
     const int smem = 4 * kTileBytes;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attn_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    if (cudaError_t e = ensure_dynamic_smem(attn_prefill_kernel, smem, &attr_done); e != cudaSuccess) return e;
     const int batch = rows / rows_per_seq;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((rows_per_seq + kBM - 1) / kBM, nq, batch);

@@ -197,12 +197,8 @@ cudaError_t launch_one(const LaunchCtx &lc, const bf16 *W, const float *x, float
                        const bf16 *gain, float eps, const ArgmaxScratch &am, int ctas_per_sm) {
     auto kern = gemv_kernel<ROWS, MODE, NORM>;
     const size_t smem = (size_t)n_in * sizeof(float);
-    static bool attr_done = false;  // per instantiation
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static unsigned long long attr_done = 0;   // per instantiation, one bit per device
+    if (cudaError_t e = ensure_dynamic_smem(kern, 200 * 1024, &attr_done); e != cudaSuccess) return e;
     const int n_groups = n_out / ROWS;
     const int cap = lc.sm_count * ctas_per_sm;
     int blocks = (n_groups + kGemvWarps - 1) / kGemvWarps;

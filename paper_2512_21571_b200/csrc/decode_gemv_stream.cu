@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     __shared__ float red[kConsumerWarps];
     __shared__ int red_i[kConsumerWarps];
     __shared__ bool is_last;
+    __shared__ int abort_s;                     // a consumer warp's wait ran out: every warp leaves at the next fold
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages;
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     const uint32_t stage_bytes = (uint32_t)p.rps * row_bytes;
 
     if (threadIdx.x == 0) {
+        abort_s = 0;
         for (int s = 0; s < S; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&full[s])));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&empty[s])), "r"(kConsumerWarps));
@@ -245,7 +247,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
         int nb = 0;
         for (int j = 0; j < p.pb; ++j) {
             if (!mbar_wait_bounded(smem_u32(&full[stage]), phase)) {
-                ok = false; done = true;
+                // give up for the whole CTA: the flag is read by every warp after the barrier below, so all of them
+                // leave the loop in the same iteration and no later barrier waits for a warp that has gone
+                ok = false;
+                *(volatile int *)&abort_s = 1;
                 if (lane == 0 && p.status) atomicExch(p.status, 16);
                 break;
             }
@@ -288,6 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
             ++nb;
         }
         consumer_sync();
+        if (*(volatile int *)&abort_s) { ok = false; break; }
         if (NORM && blk == 0) {
             float tot = 0.f;
             for (int k = 0; k < ksplit; ++k) tot += ssq[k];   // warps 0 .. ksplit-1 hold the ksplit distinct slices
@@ -372,12 +378,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
 template <int J, int MODE, bool NORM>
 cudaError_t launch_j(const LaunchCtx &lc, const StreamParams &p, int grid, size_t smem) {
     auto kern = gemv_stream_kernel<J, MODE, NORM>;
-    static bool attr_done = false;  // per instantiation
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static unsigned long long attr_done = 0;   // per instantiation, one bit per device
+    if (cudaError_t e = ensure_dynamic_smem(kern, kRingBytes, &attr_done); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
@@ -488,9 +490,11 @@ cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *
     // matrices with few stages per SM claim stage by stage so that the tail stays short
     p.claim = (stage_bytes >= 49152 || p.n_stages < 16 * lc.sm_count) ? 1 : (65536 + stage_bytes - 1) / stage_bytes;
     if (stage_bytes < 16384 && p.claim == 1) p.claim = (32768 + stage_bytes - 1) / stage_bytes;
-    p.ctr = ctr;
     const int n_runs = (p.n_stages + p.claim - 1) / p.claim;
     int grid = n_runs < lc.sm_count ? n_runs : lc.sm_count;
+    // With no more runs than CTAs every CTA takes exactly one run: dynamic claims buy nothing there, and leaving the
+    // shared counters alone means many such small launches may be in flight at once without meeting on them.
+    p.ctr = n_runs > lc.sm_count ? ctr : nullptr;
     if (mode == kGemvLogits && grid > kArgmaxMaxBlocks) grid = kArgmaxMaxBlocks;
     const size_t smem = (size_t)S * stage_bytes;
     const int J = (p.kw + 255) / 256;

@@ -668,12 +668,8 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
                       int K, int ldy, int *status, const GemmScratch *scratch) {
     using L = SmemLayout<BN, SWAP, SPLIT, KA>;
     auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static unsigned long long attr_done = 0;   // per instantiation, one bit per device
+    if (cudaError_t e = ensure_dynamic_smem(kern, L::kBytes, &attr_done); e != cudaSuccess) return e;
     CUtensorMap map_w, map_x, map_x_lo;
     GemmParams p;
     p.Y = Y; p.Y_lo = Y_lo; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status;

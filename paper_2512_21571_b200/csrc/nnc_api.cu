@@ -32,7 +32,7 @@ struct Plan {
     // offsets
     std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
-    size_t mega_layers, mega_bars, gemv_ctr, gemm_part, gemm_tickets, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
+    size_t gemv_ctr, gemm_part, gemm_tickets, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
     size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
     size_t take(size_t bytes) {
         const size_t o = total;
@@ -75,8 +75,6 @@ void make_plan(const nnc_config &c, Plan &p) {
     p.kcache = p.take(kv);
     p.vcache = p.take(kv);
     p.rope = p.take((size_t)c.max_seq * 128 * 4);
-    p.mega_layers = p.take((size_t)c.n_layers * sizeof(MegaLayer));
-    p.mega_bars = p.take(128);
     p.gemv_ctr = p.take(((size_t)c.n_layers * 4 + 2) * 16);
     p.gemm_part = p.take(c.max_tokens > 0 ? kGemmPartBytes : 0);
     p.gemm_tickets = p.take((size_t)kGemmTickets * 4);
@@ -117,8 +115,6 @@ struct nnc_model {
     bf16 *embed, *lm_head, *g_final, *kcache, *vcache;
     float *rope, *x, *qkv, *attn_out, *act, *part;
     uint32_t *tickets;
-    MegaParams mega;           // whole-step decode kernel: everything but the per-call buffers
-    bool mega_ok;              // false: use the kernel-per-phase path
     GemmScratch gemm_scratch;  // split-K partial tiles and tickets of the token-batch GEMMs
     uint32_t *gemv_ctr;  // 4 words per GEMV call site (4 per layer + lm_head): dynamic work counters, zero at rest
     ArgmaxScratch am;
@@ -195,19 +191,6 @@ int decode_b1_launches(nnc_model *m, const int32_t *tokens, float *logits, int32
     am.out = argmax;
     NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->x, logits, c.vocab, c.hidden, m->g_final, c.rms_eps, kGemvLogits, &am,
                             m->gemv_ctr + (size_t)c.n_layers * 16));
-    NNC_CUDA(m, launch_add_len(lc, m->d_len, 1));
-    return NNC_OK;
-}
-
-// The same step as one persistent kernel (decode_step_mega.cu): barrier words cleared, kernel, position + 1.
-int decode_b1_mega_launches(nnc_model *m, const int32_t *tokens, float *logits, int32_t *argmax, const LaunchCtx &lc) {
-    NNC_CUDA(m, cudaMemsetAsync(m->mega.bars, 0, 128, lc.stream));
-    MegaParams p = m->mega;
-    p.tokens = tokens;
-    p.logits = logits;
-    p.am = m->am;
-    p.am.out = argmax;
-    NNC_CUDA(m, launch_decode_mega(lc, p));
     NNC_CUDA(m, launch_add_len(lc, m->d_len, 1));
     return NNC_OK;
 }
@@ -336,8 +319,7 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         m->len = 0;
         m->taps = nullptr;
         m->launches = 0;
-        const char *pdl_env = getenv("NNC_PDL");
-        m->pdl = !(pdl_env && pdl_env[0] == '0');
+        m->pdl = c.serial_launches == 0;
 
         // ---- repack: bit moves on the device ----
         LaunchCtx lc = ctx(m, false);
@@ -361,46 +343,6 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         if (!c.tie_embeddings)
             NNC_CUDA(m, launch_copy_rows(lc, (const bf16 *)weights->lm_head, m->lm_head, c.vocab, H, 0, 1, 0, 1));
         NNC_CUDA(m, cudaMemcpyAsync(m->g_final, weights->g_final, (size_t)H * 2, cudaMemcpyDeviceToDevice, m->stream));
-
-        // ---- whole-step decode kernel: per-layer pointer table and matrix geometries ----
-        {
-            std::vector<MegaLayer> ml(c.n_layers);
-            for (int l = 0; l < c.n_layers; ++l) {
-                const LayerW &w = m->layers[l];
-                ml[l] = MegaLayer{w.wqkv, w.wo, w.wgu, w.wd, w.g_in, w.g_post, w.g_q, w.g_k,
-                                  m->kcache + (size_t)l * m->kv_layer_stride(), m->vcache + (size_t)l * m->kv_layer_stride()};
-            }
-            NNC_CUDA(m, cudaMemcpyAsync(at(p.mega_layers), ml.data(), ml.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, m->stream));
-            NNC_CUDA(m, cudaStreamSynchronize(m->stream));   // ml is a host temporary
-            MegaParams &g = m->mega;
-            memset(&g, 0, sizeof(g));
-            g.layers = (const MegaLayer *)at(p.mega_layers);
-            g.n_layers = c.n_layers;
-            bool ok = gemv_stream_geometry(m->qkvd(), H, m->sm_count, kGemvStore, &g.gq) &&
-                      gemv_stream_geometry(H, qd, m->sm_count, kGemvResidual, &g.go) &&
-                      gemv_stream_geometry(2 * I, H, m->sm_count, kGemvSwiglu, &g.gg) &&
-                      gemv_stream_geometry(H, I, m->sm_count, kGemvResidual, &g.gd) &&
-                      gemv_stream_geometry(c.vocab, H, m->sm_count, kGemvLogits, &g.gl);
-            if (ok) {
-                size_t slot = 0;
-                for (const GemvGeom *gg : {&g.gq, &g.go, &g.gg, &g.gd, &g.gl}) {
-                    const size_t b = (size_t)gg->rps * gg->K * 2;
-                    if (b > slot) slot = b;
-                }
-                g.slot_bytes = (uint32_t)((slot + 127) / 128 * 128);
-                g.embed = m->embed; g.lm_head = m->lm_head; g.g_final = m->g_final;
-                g.x = m->x; g.qkv = m->qkv; g.attn_out = m->attn_out; g.act = m->act;
-                g.part = m->part; g.tickets = m->tickets; g.d_len = m->d_len; g.rope = m->rope;
-                g.nq = c.n_q_heads; g.nkv = c.n_kv_heads; g.max_seq = c.max_seq; g.hidden = H; g.vocab = c.vocab;
-                g.n_splits = attn_decode_splits(m->sm_count, 1, c.n_kv_heads, c.max_seq);
-                g.eps = c.rms_eps;
-                g.bars = (uint32_t *)at(p.mega_bars);
-                g.status = m->d_status;
-                ok = decode_mega_supported(g, m->sm_count);
-            }
-            const char *mega_env = getenv("NNC_MEGA");
-            m->mega_ok = ok && mega_env && mega_env[0] == '1';   // opt-in: measured slower than the per-phase chain so far
-        }
 
         // ---- RoPE table: cos/sin of p * theta^(-2i/128) in double, rounded once to fp32 ----
         {
@@ -472,37 +414,24 @@ int nnc_decode_step(nnc_model *m, const int32_t *tokens, int32_t batch, float *l
     auto key = std::make_tuple((const void *)tokens, (const void *)logits, (const void *)argmax);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
-        // capture the step: first as the single whole-step kernel; if that cannot be captured or instantiated on this
-        // device (the cooperative launch is refused), as the chain of per-phase kernels
+        // capture the step once for this set of buffers
         cudaGraphExec_t exec = nullptr;
-        int64_t nodes = 0;
-        for (int attempt = 0; attempt < 2 && !exec; ++attempt) {
-            const bool mega = m->mega_ok;
-            cudaGraph_t graph = nullptr;
-            const int64_t before = m->launches;
-            NNC_CUDA(m, cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeThreadLocal));
-            LaunchCtx cap = ctx(m, m->pdl && !mega);
-            cap.stream = m->capture_stream;
-            rc = mega ? decode_b1_mega_launches(m, tokens, logits, argmax, cap) : decode_b1_launches(m, tokens, logits, argmax, cap);
-            cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
-            nodes = m->launches - before;
-            m->launches = before;
-            if (rc == NNC_OK && e == cudaSuccess) e = cudaGraphInstantiate(&exec, graph, 0);
-            if (graph) cudaGraphDestroy(graph);
-            if (rc != NNC_OK || e != cudaSuccess) {
-                exec = nullptr;
-                cudaGetLastError();
-                if (mega) {   // try again with the per-phase kernels
-                    fprintf(stderr, "nnc: whole-step decode kernel not usable here (%s%s); using the per-phase kernels\n",
-                            rc != NNC_OK ? m->err : cudaGetErrorString(e), "");
-                    m->mega_ok = false;
-                    continue;
-                }
-                if (rc != NNC_OK) return rc;
-                return fail(m, NNC_ERR_CUDA, "graph capture / instantiate failed: %s", cudaGetErrorString(e));
-            }
+        cudaGraph_t graph = nullptr;
+        const int64_t before = m->launches;
+        NNC_CUDA(m, cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeThreadLocal));
+        LaunchCtx cap = ctx(m, m->pdl);
+        cap.stream = m->capture_stream;
+        rc = decode_b1_launches(m, tokens, logits, argmax, cap);
+        cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
+        const int64_t nodes = m->launches - before;
+        m->launches = before;
+        if (rc == NNC_OK && e == cudaSuccess) e = cudaGraphInstantiate(&exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+        if (rc != NNC_OK || e != cudaSuccess) {
+            cudaGetLastError();
+            if (rc != NNC_OK) return rc;
+            return fail(m, NNC_ERR_CUDA, "graph capture / instantiate failed: %s", cudaGetErrorString(e));
         }
-        if (!exec) return fail(m, NNC_ERR_CUDA, "could not build the decode graph");
         if (m->graphs.size() >= 16) {  // callers that keep changing buffers should not leak graphs
             for (auto &g : m->graphs) cudaGraphExecDestroy(g.second.exec);
             m->graphs.clear();
@@ -762,9 +691,10 @@ int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t 
     lc.pdl = chained;
     uint32_t *ctrs = nullptr;
     if (cudaGetSymbolAddress((void **)&ctrs, g_op_gemv_ctr) != cudaSuccess) return NNC_ERR_CUDA;
-    static unsigned rotation = 0;
+    static unsigned rotation = 0;   // call sites taken in turn; atomic so that concurrent host threads get distinct ones
+    const unsigned site = __atomic_fetch_add(&rotation, 1u, __ATOMIC_RELAXED) % 8;
     cudaError_t e = launch_gemv(lc, (const bf16 *)W, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr,
-                                ctrs + 4 * (rotation++ % 8));
+                                ctrs + 4 * site);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }

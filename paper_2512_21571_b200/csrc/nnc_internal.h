@@ -33,6 +33,20 @@ inline cudaError_t launch(const LaunchCtx &lc, void (*kern)(KArgs...), dim3 grid
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of the
+// function, so a process that drives several GPUs needs it on each).  `done` is a per-kernel bit mask of devices.
+template <typename K>
+inline cudaError_t ensure_dynamic_smem(K kern, int bytes, unsigned long long *done) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (__atomic_load_n(done, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) __atomic_fetch_or(done, bit, __ATOMIC_RELEASE);
+    return e;
+}
+
 // ---- decode GEMV family (decode_gemv.cu) --------------------------------------------------------------
 enum GemvMode { kGemvStore = 0, kGemvResidual = 1, kGemvSwiglu = 2, kGemvLogits = 3 };
 
@@ -62,34 +76,6 @@ struct GemvGeom {
     int ksplit, kw, rps, n_stages, J;
 };
 bool gemv_stream_geometry(int n_out, int n_in, int sm_count, int mode, GemvGeom *out);
-
-// ---- whole-step decode kernel (decode_step_mega.cu) ----------------------------------------------------
-struct MegaLayer {
-    const bf16 *wqkv, *wo, *wgu, *wd, *g_in, *g_post, *g_q, *g_k;
-    bf16 *kc, *vc;
-};
-struct MegaParams {
-    const MegaLayer *layers;   // DEVICE array, n_layers entries
-    int n_layers;
-    GemvGeom gq, go, gg, gd, gl;   // QKV, O, gate/up, down, lm_head
-    const bf16 *embed, *lm_head, *g_final;
-    const int32_t *tokens;     // [1]
-    float *x, *qkv, *attn_out, *act, *logits;
-    ArgmaxScratch am;          // am.out == null: no arg-max
-    float *part;
-    uint32_t *tickets;
-    const int32_t *d_len;
-    const float *rope;
-    int nq, nkv, max_seq, n_splits, hidden, vocab;
-    float eps;
-    uint32_t *bars;            // 32 words of grid-barrier state (counters, release word, abort word), zero at launch
-    int *status;
-    int stages;                // ring depth
-    uint32_t slot_bytes;       // ring slot size (largest stage of the step)
-};
-// false: shape outside what the whole-step kernel covers (the caller uses the kernel-per-phase path)
-bool decode_mega_supported(const MegaParams &p, int sm_count);
-cudaError_t launch_decode_mega(const LaunchCtx &lc, const MegaParams &p);
 
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,

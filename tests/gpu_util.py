@@ -26,3 +26,9 @@ def rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
     a, b = a.double().cpu(), b.double().cpu()
     a, b = a.reshape(-1, a.shape[-1]), b.reshape(-1, b.shape[-1])
     return ((a - b).norm(dim=-1) / b.norm(dim=-1)).max().item()
+
+
+def split_bf16(x: torch.Tensor):
+    """fp32 -> (hi, lo) bf16 pair with hi + lo ~ x to 16 mantissa bits: test input for the two-term GEMM operand."""
+    hi = x.to(torch.bfloat16)
+    return hi, (x - hi.float()).to(torch.bfloat16)

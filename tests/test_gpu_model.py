@@ -187,27 +187,3 @@ def test_host_variants_and_errors(oracle_mod):
     m.set_length(0)
     m.prefill(torch.tensor([[-5, shape.vocab + 7, 3]], dtype=torch.int32, device="cuda"))
     assert m.device_status() == 0
-
-
-def test_whole_step_kernel_matches_the_per_phase_chain(oracle_mod, monkeypatch):
-    """NNC_MEGA=1 runs the decode step as one persistent kernel (grid barriers between phases).  It reuses the
-    arithmetic of the per-phase kernels, so logits and arg-max must be bit-identical, step after step."""
-    shape = synth.SHAPES["tiny-untied"]
-    toks = synth.prompt_tokens(shape, 21, 8).cuda().view(1, 8)
-    tok = torch.tensor([5], dtype=torch.int32, device="cuda")
-    runs = []
-    for mega in ("0", "1"):
-        monkeypatch.setenv("NNC_MEGA", mega)
-        m, o, w = make_pair(oracle_mod, shape, 21, max_seq=64, max_tokens=8)
-        m.prefill(toks, want_logits=False)
-        logits = torch.empty(shape.vocab, device="cuda")
-        am = torch.zeros(1, dtype=torch.int32, device="cuda")
-        out = []
-        for _ in range(5):
-            m.decode_step(tok, logits, am)
-            out.append((logits.clone(), int(am.item())))
-        assert m.device_status() == 0
-        runs.append(out)
-        m.close(); o.close()
-    for (la, aa), (lb, ab) in zip(*runs):
-        assert torch.equal(la, lb) and aa == ab

@@ -5,6 +5,7 @@ import math
 import pytest
 import torch
 
+from gpu_util import split_bf16
 from paper_2512_21571_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -125,7 +126,7 @@ def test_gemm_split_activations_recover_fp32_inputs(nnc, oracle_mod, T, N, K):
     (the oracle's matmul on the unrounded X) to ~2^-16, on both operand assignments (T <= 128 and T > 128)."""
     X = synth.normal(7, 1, (T, K), 1.0, torch.float32, "cuda")
     W = _w(7, 2, (N, K))
-    hi, lo = nnc.split_bf16(X)
+    hi, lo = split_bf16(X)
     Y = nnc.op_gemm(hi, W, X_lo=lo)
     rows = sorted(set([0, T - 1, T // 2]))
     want = oracle_mod.matmul(W.cpu(), X[rows].cpu())
@@ -155,7 +156,7 @@ def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
     run, scratch flags left at zero."""
     X = synth.normal(8, 1, (T, K), 1.0, torch.float32, "cuda")
     W = _w(8, 2, (N, K))
-    hi, lo = nnc.split_bf16(X)
+    hi, lo = split_bf16(X)
     scratch = torch.zeros(16384 + (32 << 20), dtype=torch.uint8, device="cuda")
     Y = nnc.op_gemm_splitk(hi, W, scratch, X_lo=lo)
     Y2 = nnc.op_gemm_splitk(hi, W, scratch, X_lo=lo)
