@@ -206,14 +206,16 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
                        int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_ctx, void *scratch,
                        void *cuda_stream);
 
-/* Causal attention of the prompt phase for T new tokens per sequence.
+/* Causal attention of the prompt phase for T new tokens per sequence (tcgen05 tensor cores; the score and
+ * probability tile stays in tensor memory between the two products, cf. the pass-through layout of Section 3.1.2).
  *   qkv fp32 [batch * T][(n_q_heads + 2 n_kv_heads) * 128]: only the query heads are read (already normalised and
  *   rotated);  kcache, vcache bf16 [batch][n_kv_heads][max_seq][128] must already hold the new tokens' K/V at
- *   positions n_past .. n_past + T - 1;  the query of token s attends to positions 0 .. n_past + s.
- *   out (and out_lo, NULL or the bf16 rounding residual): bf16 [batch * T][n_q_heads * 128].
- *   n_past_dev: DEVICE int32 holding n_past. */
+ *   positions n_past .. n_past + T - 1;  the query of token s attends to positions 0 .. n_past + s.  Cache rows at
+ *   positions >= n_past + T are never read (they may hold anything).
+ *   out (and out_lo, NULL or the bf16 rounding residual): bf16 [batch * T][n_q_heads * 128], 16-byte aligned.
+ *   n_past: cached positions before these tokens, a host value; n_past + T > max_seq returns NNC_ERR_CAPACITY. */
 int nnc_op_attn_prefill(const float *qkv, const void *kcache, const void *vcache, void *out, void *out_lo, int32_t batch,
-                        int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, const int32_t *n_past_dev,
+                        int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_past,
                         void *cuda_stream);
 
 /* The same operation for callers that cannot allocate device memory (the paper has no counterpart: this is a

@@ -73,7 +73,7 @@ EXPORTS = {
     "nnc_op_attn_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "nnc_op_attn_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
-                                      C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+                                      C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "nnc_op_attn_decode_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
 }
@@ -314,8 +314,7 @@ def op_attn_prefill(qkv: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tenso
     batch, nkv, max_seq, _ = kcache.shape
     out = torch.empty(batch * T, n_q_heads * 128, dtype=torch.bfloat16, device="cuda")
     out_lo = torch.empty_like(out)
-    past = torch.tensor([n_past], dtype=torch.int32, device="cuda")
     _ok(lib.nnc_op_attn_prefill(_dev(qkv, torch.float32), _dev(kcache, torch.bfloat16), _dev(vcache, torch.bfloat16),
-                                out.data_ptr(), out_lo.data_ptr(), batch, T, n_q_heads, nkv, max_seq, past.data_ptr(),
+                                out.data_ptr(), out_lo.data_ptr(), batch, T, n_q_heads, nkv, max_seq, n_past,
                                 _stream_ptr()), "nnc_op_attn_prefill")
     return out, out_lo

@@ -1,0 +1,414 @@
+// Causal attention of the prompt phase on the 5th-generation tensor cores: the query at position p attends to
+// cache positions 0..p of its sequence.  K and V are read from the bf16 cache, which already holds the new tokens.
+//
+// The score / probability tile never leaves the SM between the two products -- the form the paper's
+// "MatMul -> Exp -> MatMul" pass-through layout takes here (Section 3.1.2, Eq. 1): S = Q K^T is accumulated in
+// tensor memory, the softmax warps read it with tcgen05.ld, and write the probabilities back over it as the bf16
+// A operand of O += P V, which tcgen05.mma reads straight from tensor memory.
+//
+// One CTA per (128 query rows, query head, sequence), 192 threads:
+//   warp 0      TMA producer: K and V tiles of 128 cache positions (two 128B-swizzled boxes of 64 head-dimension
+//               elements each) into a two-stage shared-memory ring.  The tensor map's position extent is the number
+//               of valid cache rows, so rows past the end arrive as zeros (0 * stale bits would not be 0).
+//   warp 1      MMA issuer (one lane): S[j&1] = Q K_j^T into one of two score buffers, so the product of tile j+1
+//               runs while the softmax warps work on tile j; then O += P_j V_j with V as an MN-major operand (the
+//               cache row is [position][head dim], contraction over positions).
+//   warps 2-5   one thread per query row: load Q (fp32, already normalised and rotated), scale to log2 units and
+//               write it to shared memory in the swizzled K-major layout; per tile: scores -> mask (diagonal tiles)
+//               -> exp2 -> probabilities; finally O / l to the output.
+// Q and P are fed as two bf16 terms (value + rounding residual) multiplied into the same accumulator: a single
+// bf16 term costs 2^-9 per operand, which the parity tolerance of deep models does not allow.
+// Online softmax with a lazy maximum: the running maximum m only moves (and O is rescaled in tensor memory) when a
+// tile's maximum exceeds it by more than 2^8; probabilities then stay below 256, which fp32 sums and the bf16
+// pair hold without loss.  The result is the exact softmax whatever m is.
+// Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains and frees its tensor memory.
+#include "tc_common.cuh"
+
+namespace nnc {
+
+namespace {
+
+constexpr int kQM = 128;                 // query rows per CTA
+constexpr int kKN = 128;                 // cache positions per tile
+constexpr int kPfThreads = 192;
+constexpr int kSlab = 128 * 128;         // bytes of a [128 rows][64 x 16 bit] swizzled slab
+constexpr int kTile = 2 * kSlab;         // [128][128] 16-bit tile = two slabs (head-dimension halves)
+constexpr int kPfSmem = 6 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   // Q hi, Q lo, 2 x (K, V)
+constexpr uint32_t kColS = 0, kColO = 256, kTmemCols = 512;
+constexpr float kLazyMax = 8.f;          // log2 units
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+
+// tcgen05.mma with the A operand in tensor memory (K-major, two 16-bit elements per 32-bit column)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Shared-memory descriptor of an MN-major 16-bit operand under the 128-byte swizzle: 64 elements (128 bytes) are
+// contiguous along MN, the next 64 follow `lbo` bytes later; along K, rows are 128 bytes apart and groups of 8 rows
+// 1024 bytes.  That is exactly a [position][64] TMA box of cache rows, with the head-dimension halves one slab apart.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr, uint32_t lbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+struct PfParams {
+    const float *qkv;   // [batch * T][row_stride]: query heads first
+    int row_stride;     // floats per token row = (nq + 2 nkv) * 128
+    void *out, *out_lo; // [batch * T][nq * 128]: bf16 value (+ residual, nullable), or fp16
+    int T, n_past, nq, nkv;
+    int *status;
+};
+
+// OUT_FP16: the output is one fp16 matrix (saturating) instead of a bf16 value + residual pair
+template <bool OUT_FP16>
+__global__ void __launch_bounds__(kPfThreads, 1)
+attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_hi = base, q_lo = base + kTile;
+    auto k_tile = [&](int s) { return base + 2u * kTile + (uint32_t)s * 2u * kTile; };
+    auto v_tile = [&](int s) { return k_tile(s) + (uint32_t)kTile; };
+    const uint32_t bars = base + 6u * kTile;
+    const uint32_t q_ready = bars;
+    auto k_full = [&](int s) { return bars + 8u * (1 + s); };
+    auto v_full = [&](int s) { return bars + 8u * (3 + s); };
+    auto s_full = [&](int s) { return bars + 8u * (5 + s); };
+    auto p_full = [&](int s) { return bars + 8u * (7 + s); };
+    auto pv_done = [&](int s) { return bars + 8u * (9 + s); };
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &abort_s;
+    const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;   // longest rows first
+    const int h = blockIdx.y, seq = blockIdx.z;
+    const int G = p.nq / p.nkv, jkv = h / G;
+    const int q0 = qt * kQM;
+    const int n_valid = p.n_past + p.T;
+    const int n_keys = min(p.n_past + q0 + kQM, n_valid);   // cache positions the last row of this tile may see
+    const int n_tiles = (n_keys + kKN - 1) / kKN;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(q_ready, 128);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(k_full(s), 1); mbar_init(v_full(s), 1); mbar_init(s_full(s), 1);
+            mbar_init(p_full(s), 128); mbar_init(pv_done(s), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        if (lane == 0) {   // ---------------- TMA producer ----------------
+            pdl_wait();    // the cache rows of the new tokens come from the preceding kernel
+            const int z = seq * p.nkv + jkv;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int s = j & 1, u = j >> 1;
+                if (j >= 2 && !mbar_wait(pv_done(s), (uint32_t)((u - 1) & 1), abort_flag, p.status, 21)) break;
+                mbar_expect_tx(k_full(s), kTile);
+                tma_load_3d(k_tile(s), &map_k, k_full(s), 0, j * kKN, z);
+                tma_load_3d(k_tile(s) + kSlab, &map_k, k_full(s), 64, j * kKN, z);
+                mbar_expect_tx(v_full(s), kTile);
+                tma_load_3d(v_tile(s), &map_v, v_full(s), 0, j * kKN, z);
+                tma_load_3d(v_tile(s) + kSlab, &map_v, v_full(s), 64, j * kKN, z);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {   // ---------------- MMA issuer ----------------
+            constexpr uint32_t idesc_qk = make_idesc(kKN, false, false);
+            constexpr uint32_t idesc_pv = make_idesc(kHeadDim, false, true);
+            bool ok = mbar_wait(q_ready, 0u, abort_flag, p.status, 22);
+            tc_fence_after();
+            auto issue_qk = [&](int j) -> bool {
+                const int s = j & 1, u = j >> 1;
+                if (!mbar_wait(k_full(s), (uint32_t)(u & 1), abort_flag, p.status, 23)) return false;
+                if (j >= 2 && !mbar_wait(pv_done(s), (uint32_t)((u - 1) & 1), abort_flag, p.status, 24)) return false;
+                tc_fence_after();
+                const uint32_t d = tmem_base + kColS + (uint32_t)s * kKN;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {   // 16 head-dimension elements per instruction
+                    const uint32_t off = (uint32_t)(ks >> 2) * kSlab + (uint32_t)(ks & 3) * 32u;
+                    const uint64_t b = make_smem_desc(k_tile(s) + off);
+                    umma_bf16(d, make_smem_desc(q_hi + off), b, idesc_qk, ks != 0);
+                    umma_bf16(d, make_smem_desc(q_lo + off), b, idesc_qk, 1u);
+                }
+                umma_commit(s_full(s));
+                return true;
+            };
+            if (ok) ok = issue_qk(0);
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                if (j + 1 < n_tiles && !issue_qk(j + 1)) break;
+                const int s = j & 1, u = j >> 1;
+                if (!mbar_wait(p_full(s), (uint32_t)(u & 1), abort_flag, p.status, 25)) break;
+                if (!mbar_wait(v_full(s), (uint32_t)(u & 1), abort_flag, p.status, 26)) break;
+                tc_fence_after();
+                const uint32_t d = tmem_base + kColO;
+                const uint32_t pa = tmem_base + kColS + (uint32_t)s * kKN;   // P value in columns 0..63, residual in 64..127
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {   // 16 cache positions per instruction
+                    const uint64_t b = make_smem_desc_mn(v_tile(s) + (uint32_t)ks * 2048u, kSlab);
+                    umma_bf16_ts(d, pa + (uint32_t)ks * 8u, b, idesc_pv, (j != 0) || (ks != 0));
+                    umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
+                }
+                umma_commit(pv_done(s));
+            }
+        }
+    } else {   // ---------------- softmax warps 2..5: one thread per query row ----------------
+        const int quarter = warp & 3;                    // the TMEM lane quarter this warp may touch
+        const int r = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int tok = q0 + r;
+        const bool valid = tok < p.T;
+        const int pos = p.n_past + tok;                  // absolute position of this row's query
+        pdl_wait();
+        {   // Q -> shared memory, K-major with the 128-byte swizzle (16-byte chunk index XOR row % 8), value + residual
+            const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
+            const float *src = p.qkv + ((size_t)seq * p.T + (size_t)min(tok, p.T - 1)) * p.row_stride + (size_t)h * kHeadDim;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                float4 a = reinterpret_cast<const float4 *>(src)[2 * c], b = reinterpret_cast<const float4 *>(src)[2 * c + 1];
+                if (!valid) { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+                const float f[8] = {a.x * qscale, a.y * qscale, a.z * qscale, a.w * qscale,
+                                    b.x * qscale, b.y * qscale, b.z * qscale, b.w * qscale};
+                uint4 hi, lo;
+                hi.x = pack_bf16x2(f[0], f[1]); lo.x = pack_bf16x2(f[0] - bf16_lo(hi.x), f[1] - bf16_hi(hi.x));
+                hi.y = pack_bf16x2(f[2], f[3]); lo.y = pack_bf16x2(f[2] - bf16_lo(hi.y), f[3] - bf16_hi(hi.y));
+                hi.z = pack_bf16x2(f[4], f[5]); lo.z = pack_bf16x2(f[4] - bf16_lo(hi.z), f[5] - bf16_hi(hi.z));
+                hi.w = pack_bf16x2(f[6], f[7]); lo.w = pack_bf16x2(f[6] - bf16_lo(hi.w), f[7] - bf16_hi(hi.w));
+                const uint32_t off = (uint32_t)(c >> 3) * kSlab + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                sts128(q_hi + off, hi);
+                sts128(q_lo + off, lo);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes, async-proxy (MMA) reads
+            mbar_arrive(q_ready);
+        }
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_tiles; ++j) {
+            const int s = j & 1, u = j >> 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(s_full(s), (uint32_t)(u & 1), abort_flag, p.status, 27));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t ts = tmem_base + lane_addr + kColS + (uint32_t)s * kKN;
+            float sv[128];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t t[32];
+                tmem_ld32(ts + 32u * i, t);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) sv[32 * i + e] = __uint_as_float(t[e]);
+            }
+            const int k0 = j * kKN;
+            if (k0 + kKN - 1 > p.n_past + q0) {   // the tile reaches past the first row's position: causal mask
+#pragma unroll
+                for (int e = 0; e < 128; ++e)
+                    if (k0 + e > pos) sv[e] = -INFINITY;
+            }
+            float m_tile = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 128; ++e) m_tile = fmaxf(m_tile, sv[e]);
+            if (j == 0) {
+                m_used = m_tile;   // finite: position 0 is visible to every row
+            } else {
+                const bool need = m_tile > m_used + kLazyMax;
+                if (__any_sync(0xffffffffu, need)) {
+                    // O is rescaled in tensor memory; the product of the previous tile must have landed first
+                    ok = __all_sync(0xffffffffu, mbar_wait(pv_done((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, p.status, 28));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float m_new = need ? m_tile : m_used;
+                    const float alpha = exp2f(m_used - m_new);   // 1 for the rows that keep their maximum
+                    const uint32_t to = tmem_base + lane_addr + kColO;
+#pragma unroll 1
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t t[32];
+                        tmem_ld32(to + 32u * i, t);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) t[e] = __float_as_uint(__uint_as_float(t[e]) * alpha);
+                        tmem_st32(to + 32u * i, t);
+                    }
+                    tmem_wait_st();
+                    l *= alpha;
+                    m_used = m_new;
+                }
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int e = 0; e < 128; ++e) { sv[e] = exp2f(sv[e] - m_used); sum += sv[e]; }
+            l += sum;
+            // P over S: value pairs in columns 0..63, residual pairs in columns 64..127 (two positions per column)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t ph[16], pl[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const float a = sv[32 * i + 2 * e], b = sv[32 * i + 2 * e + 1];
+                    ph[e] = pack_bf16x2(a, b);
+                    pl[e] = pack_bf16x2(a - bf16_lo(ph[e]), b - bf16_hi(ph[e]));
+                }
+                tmem_st16(ts + 16u * i, ph);
+                tmem_st16(ts + 64u + 16u * i, pl);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(p_full(s));
+        }
+        // ---- O / l -> output ----
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done((n_tiles - 1) & 1), (uint32_t)(((n_tiles - 1) >> 1) & 1), abort_flag, p.status, 29));
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l;
+            const uint32_t to = tmem_base + lane_addr + kColO;
+            const size_t oi = ((size_t)seq * p.T + (size_t)tok) * p.nq * kHeadDim + (size_t)h * kHeadDim;
+#pragma unroll 1
+            for (int i = 0; i < 4; ++i) {
+                uint32_t t[32];
+                tmem_ld32(to + 32u * i, t);
+                if (!valid) continue;
+                if (OUT_FP16) {
+                    uint32_t o[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        o[e] = pack_f16x2_sat(__uint_as_float(t[2 * e]) * inv, __uint_as_float(t[2 * e + 1]) * inv);
+                    uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__half *>(p.out) + oi + 32 * i);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+                } else {
+                    uint32_t o[16], ol[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float a = __uint_as_float(t[2 * e]) * inv, b = __uint_as_float(t[2 * e + 1]) * inv;
+                        o[e] = pack_bf16x2(a, b);
+                        ol[e] = pack_bf16x2(a - bf16_lo(o[e]), b - bf16_hi(o[e]));
+                    }
+                    uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<bf16 *>(p.out) + oi + 32 * i);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+                    if (p.out_lo) {
+                        uint4 *dl = reinterpret_cast<uint4 *>(reinterpret_cast<bf16 *>(p.out_lo) + oi + 32 * i);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) dl[e] = make_uint4(ol[4 * e], ol[4 * e + 1], ol[4 * e + 2], ol[4 * e + 3]);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----
+    __syncwarp();
+    if (*abort_flag && threadIdx.x == 0) {
+        // let copies that are still in flight land before the shared memory is released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// bf16 cache of one layer as a 3-D tensor [heads = batch * nkv][positions][128]; only the first n_valid positions of
+// every head are inside the tensor, so the rest of a box arrives as zeros
+bool make_cache_map(CUtensorMap *map, const bf16 *cache, int heads, int n_valid, int max_seq) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_valid, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)max_seq * kHeadDim * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kKN, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16 *>(cache), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool OUT_FP16>
+cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensorMap &mv, const PfParams &p, dim3 grid) {
+    auto kern = attn_prefill_tc_kernel<OUT_FP16>;
+    static unsigned long long attr_done = 0;   // per instantiation, one bit per device
+    if (cudaError_t e = ensure_dynamic_smem(kern, kPfSmem, &attr_done); e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kPfThreads);
+    cfg.dynamicSmemBytes = kPfSmem;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = lc.pdl ? 1 : 0;
+    if (lc.launches) ++*lc.launches;
+    return cudaLaunchKernelEx(&cfg, kern, mk, mv, p);
+}
+
+}  // namespace
+
+// rows = batch * rows_per_seq new tokens, the token of row s * rows_per_seq + i sitting at position n_past + i of
+// sequence s; the cache must already hold their K/V.  n_past is a host value: it sizes the tensor maps.
+cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
+                                const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
+                                int n_past) {
+    const int batch = rows / rows_per_seq, T = rows_per_seq;
+    if (T <= 0 || batch <= 0 || n_past < 0 || n_past + T > max_seq || nq % nkv) return cudaErrorInvalidValue;
+    if (((uintptr_t)qkv | (uintptr_t)kcache | (uintptr_t)vcache | (uintptr_t)out | (uintptr_t)out_lo) & 15) return cudaErrorInvalidValue;
+    CUtensorMap mk, mv;
+    if (!make_cache_map(&mk, kcache, batch * nkv, n_past + T, max_seq) || !make_cache_map(&mv, vcache, batch * nkv, n_past + T, max_seq))
+        return cudaErrorInvalidValue;
+    PfParams p;
+    p.qkv = qkv; p.row_stride = (nq + 2 * nkv) * kHeadDim; p.out = out; p.out_lo = out_lo;
+    p.T = T; p.n_past = n_past; p.nq = nq; p.nkv = nkv; p.status = lc.status;
+    const dim3 grid((T + kQM - 1) / kQM, nq, batch);
+    return out_fp16 ? launch_pf<true>(lc, mk, mv, p, grid) : launch_pf<false>(lc, mk, mv, p, grid);
+}
+
+}  // namespace nnc

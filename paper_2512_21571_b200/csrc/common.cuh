@@ -22,6 +22,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return (uint32_t)f32_to_bf16_bits(lo) | ((uint32_t)f32_to_bf16_bits(hi) << 16);
 }
 
+// two floats -> packed fp16 pair (lo in bits 0..15), round to nearest even, saturating at +-65504 instead of infinity
+__device__ __forceinline__ uint32_t pack_f16x2_sat(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
 // 16-byte read-only streaming load: weights and cache lines are used once per step, keep them out of L1.
 __device__ __forceinline__ uint4 ldg_stream(const void *p) {
     uint4 v;

@@ -86,6 +86,8 @@ qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, 
 
 // out[i][:] = bf16(RMSNorm(x[first + i*step][:]; gain)); one block per output row.  If out_lo is given it
 // receives the bf16 rounding residual (value - float(out)), so that out + out_lo carries 16 mantissa bits.
+// F16: out receives fp16 values instead (one term, saturating at +-65504).
+template <bool F16>
 __global__ void __launch_bounds__(256)
 rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out,
                     bf16 *__restrict__ out_lo, int H, float eps, int first, int step) {
@@ -123,6 +125,12 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
         const float y0 = v.x * inv * bf16_lo(g.x), y1 = v.y * inv * bf16_hi(g.x);
         const float y2 = v.z * inv * bf16_lo(g.y), y3 = v.w * inv * bf16_hi(g.y);
         uint2 o;
+        if (F16) {
+            o.x = pack_f16x2_sat(y0, y1);
+            o.y = pack_f16x2_sat(y2, y3);
+            dst[i] = o;
+            return;
+        }
         o.x = pack_bf16x2(y0, y1);
         o.y = pack_bf16x2(y2, y3);
         dst[i] = o;
@@ -171,8 +179,9 @@ cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows
 }
 
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
-                                int H, float eps, int first, int step) {
-    return launch(lc, rmsnorm_rows_kernel, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
+                                int H, float eps, int first, int step, bool out_f16) {
+    if (out_f16) return launch(lc, rmsnorm_rows_kernel<true>, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
+    return launch(lc, rmsnorm_rows_kernel<false>, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
 }
 
 cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n) {

@@ -11,12 +11,12 @@
 // Two operand assignments share the code: tokens on the M side (prefill; weights are the N operand, BN=256)
 // or weights on the M side ("swap", used when there are few tokens, e.g. a decode batch of 32: weights fill
 // the 128 TMEM lanes and the tokens are the narrow N operand, so no tensor-core work is wasted on padding).
+// Operand types: bf16 (activations optionally as value + rounding residual, two MMAs per weight tile) or fp16 (one
+// term; the weights are then an fp16 copy scaled by a power of two, undone by `out_scale` in the epilogue).  A and B
+// of one tcgen05.mma always have the same type.
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA raises an abort flag, records a
 // status word for the host, drains and frees its TMEM.
-#include <cuda.h>
-
-#include "common.cuh"
-#include "nnc_internal.h"
+#include "tc_common.cuh"
 
 namespace nnc {
 
@@ -25,103 +25,6 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kGemmThreads = 192;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false if the limit ran out or another role aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          int code) {
-    unsigned long long t0 = 0;
-    for (uint32_t spin = 0;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 1023u) == 1023u) {
-            if (*abort_flag) return false;
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(status, code);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes (64 elements) with the
-// 128-byte swizzle TMA applied: 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1,
-// layout type 2 (128B swizzle).  Advancing K by 16 elements inside the swizzle atom adds 32 bytes to the start.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;            // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset
-    d |= (uint64_t)1 << 46;            // descriptor version
-    d |= (uint64_t)2 << 61;            // 128-byte swizzle
-    return d;
-}
-
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc(int bn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-}
 
 struct GemmParams {
     void *Y;          // output
@@ -132,6 +35,7 @@ struct GemmParams {
     int stream;          // 1: the (tile, K stage) space is cut into one contiguous range per CTA (SWAP only)
     float *part;         // stream: fp32 partial tiles [CTA][first / last segment][BN / 32][8][128 rows][4]
     uint32_t *tickets;   // stream: one "piece parked" flag per partial-tile slot, zero at rest
+    const float *out_scale;   // DEVICE scalar multiplied into every accumulator before the epilogue (nullable = 1)
     int *status;
 };
 
@@ -202,7 +106,8 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + 
 // EPI: 0 fp32 store, 1 bf16 store, 2 fp32 accumulate (Y += D), 3 SwiGLU on interleaved gate/up weight rows -> bf16
 // SPLIT: the activations come as two bf16 matrices (value and rounding residual); both are multiplied with the
 // same weight tile into the same accumulator, which restores ~16 mantissa bits on the activation side.
-template <int BN, bool SWAP, int EPI, bool SPLIT, int KA>
+// F16: operands are fp16 (single term) and the SwiGLU epilogue writes one fp16 matrix (saturating at +-65504).
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_x_lo, GemmParams p) {
@@ -281,7 +186,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else if (warp == 1) {
         if (lane == 0) {  // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc = make_idesc(BN);
+            constexpr uint32_t idesc = make_idesc(BN, F16);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -332,6 +237,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const unsigned long long trk0 = NNC_TRACE_NOW();
         (void)trk0;
         pdl_wait();
+        const float osc = p.out_scale ? __ldg(p.out_scale) : 1.f;
         int acc = 0;
         uint32_t acc_phase = 0;
         // SWAP stores: row m = weight row, columns = tokens n0 .. n0 + 31; a warp stores 32 consecutive weight rows per token
@@ -511,7 +417,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 }
                             }
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i]);
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i] * osc);
                             const unsigned long long tr2 = NNC_TRACE_NOW();
                             (void)tr2;
                             store_swap(r, m, nt * BN + c0);
@@ -537,6 +443,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                if (p.out_scale) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * osc);
+                }
                 const int n0 = nt * BN + c0;
                 if (!SWAP) {
                     // row m = token, columns n0.. = weight rows: contiguous per thread
@@ -551,8 +461,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 for (int i = 0; i < 8; ++i) {
                                     const float a0 = silu_mul(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
                                     const float a1 = silu_mul(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-                                    o[i] = pack_bf16x2(a0, a1);
-                                    ol[i] = pack_bf16x2(a0 - bf16_lo(o[i]), a1 - bf16_hi(o[i]));
+                                    if (F16) {
+                                        o[i] = pack_f16x2_sat(a0, a1);
+                                        ol[i] = 0u;
+                                    } else {
+                                        o[i] = pack_bf16x2(a0, a1);
+                                        ol[i] = pack_bf16x2(a0 - bf16_lo(o[i]), a1 - bf16_hi(o[i]));
+                                    }
                                 }
                                 reinterpret_cast<uint4 *>(y)[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 reinterpret_cast<uint4 *>(y)[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -564,9 +479,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 for (int i = 0; i < 16; ++i)
                                     if (n0 + 2 * i + 1 < p.N) {
                                         const float a = silu_mul(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
-                                        const bf16 hi = __float2bfloat16_rn(a);
-                                        y[i] = hi;
-                                        if (yl) yl[i] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                                        if (F16) {
+                                            reinterpret_cast<uint16_t *>(y)[i] = (uint16_t)(pack_f16x2_sat(a, 0.f) & 0xffffu);
+                                        } else {
+                                            const bf16 hi = __float2bfloat16_rn(a);
+                                            y[i] = hi;
+                                            if (yl) yl[i] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                                        }
                                     }
                             }
                         } else if (EPI == 1) {
@@ -634,48 +553,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
 // ---- host side ----------------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // bf16 matrix [rows][K], K contiguous; box = 64 columns (128 bytes) x box_rows, 128-byte swizzle, zero fill
-bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows) {
+bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows, bool fp16 = false) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+    return enc(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool SWAP, int EPI, bool SPLIT, int KA>
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16 = false>
 cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
-                      int K, int ldy, int *status, const GemmScratch *scratch) {
+                      int K, int ldy, int *status, const GemmScratch *scratch, const float *out_scale = nullptr) {
     using L = SmemLayout<BN, SWAP, SPLIT, KA>;
-    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA>;
+    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA, F16>;
     static unsigned long long attr_done = 0;   // per instantiation, one bit per device
     if (cudaError_t e = ensure_dynamic_smem(kern, L::kBytes, &attr_done); e != cudaSuccess) return e;
     CUtensorMap map_w, map_x, map_x_lo;
     GemmParams p;
-    p.Y = Y; p.Y_lo = Y_lo; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status;
+    p.Y = Y; p.Y_lo = Y_lo; p.T = T; p.N = N; p.K = K; p.ldy = ldy; p.status = status; p.out_scale = out_scale;
     const int w_box = SWAP ? kBM : BN, x_box = SWAP ? BN : kBM;
-    if (!make_map(&map_w, W, N, K, w_box) || !make_map(&map_x, X, T, K, x_box)) return cudaErrorInvalidValue;
-    if (!make_map(&map_x_lo, SPLIT ? X_lo : X, T, K, x_box)) return cudaErrorInvalidValue;
+    if (!make_map(&map_w, W, N, K, w_box, F16) || !make_map(&map_x, X, T, K, x_box, F16)) return cudaErrorInvalidValue;
+    if (!make_map(&map_x_lo, SPLIT ? X_lo : X, T, K, x_box, F16)) return cudaErrorInvalidValue;
     if (!SWAP) {
         p.m_tiles = (T + kBM - 1) / kBM;
         p.n_tiles = (N + BN - 1) / BN;
@@ -728,7 +631,12 @@ cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, cons
 
 template <int EPI, bool SPLIT>
 cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
-                     int K, int ldy, int *status, const GemmScratch *sc) {
+                     int K, int ldy, int *status, const GemmScratch *sc, bool f16, const float *out_scale) {
+    if (f16) {   // fp16 operands: the prompt-phase form only (tokens on the M side, one term)
+        if (SPLIT || T <= 128) return cudaErrorInvalidValue;
+        return launch_tc_ka<256, false, EPI, false, 1, true>(lc, X, nullptr, W, Y, Y_lo, T, N, K, ldy, status, sc, out_scale);
+    }
+    if (out_scale) return cudaErrorInvalidValue;
     if (T <= 32) return launch_tc<32, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
     if (T <= 64) return launch_tc<64, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
     if (T <= 128) return launch_tc<128, true, EPI, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
@@ -737,12 +645,12 @@ cudaError_t dispatch(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const
 
 template <bool SPLIT>
 cudaError_t dispatch_epi(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                         int N, int K, int ldy, int epi, int *status, const GemmScratch *sc) {
+                         int N, int K, int ldy, int epi, int *status, const GemmScratch *sc, bool f16, const float *out_scale) {
     switch (epi) {
-        case kEpiStoreF32: return dispatch<0, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
-        case kEpiStoreBf16: return dispatch<1, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
-        case kEpiAccumF32: return dispatch<2, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
-        case kEpiSwigluBf16: return dispatch<3, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc);
+        case kEpiStoreF32: return dispatch<0, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc, f16, out_scale);
+        case kEpiStoreBf16: return dispatch<1, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc, f16, out_scale);
+        case kEpiAccumF32: return dispatch<2, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc, f16, out_scale);
+        case kEpiSwigluBf16: return dispatch<3, SPLIT>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, sc, f16, out_scale);
     }
     return cudaErrorInvalidValue;
 }
@@ -751,17 +659,19 @@ cudaError_t dispatch_epi(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
 
 bool gemm_tc_available() { return get_encode() != nullptr; }
 
-// Y[T][*] (row stride ldy) = epilogue((X + X_lo)[T][K] * W[N][K]^T).  Operands 16-byte aligned, K % 64 == 0.
+// Y[T][*] (row stride ldy) = epilogue(out_scale * (X + X_lo)[T][K] * W[N][K]^T).  Operands 16-byte aligned, K % 64 == 0.
+// f16: X and W hold fp16 instead of bf16 (T > 128, no X_lo); the SwiGLU epilogue then writes fp16.
 cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch) {
+                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch, bool f16,
+                        const float *out_scale) {
     if (T <= 0 || N <= 0 || K <= 0 || K % kBK != 0 || N % 8 != 0) return cudaErrorInvalidValue;
     if (((uintptr_t)X | (uintptr_t)X_lo | (uintptr_t)W | (uintptr_t)Y | (uintptr_t)Y_lo) & 15) return cudaErrorInvalidValue;
     // the epilogue stores 16-byte vectors per output row: the row pitch must keep them aligned
     const bool out_bf16 = epi == kEpiStoreBf16 || epi == kEpiSwigluBf16;
     if (ldy % (out_bf16 ? 8 : 4) != 0) return cudaErrorInvalidValue;
     if (epi == kEpiSwigluBf16 && N % 16 != 0) return cudaErrorInvalidValue;   // outputs leave in chunks of 8
-    return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch)
-                : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch);
+    return X_lo ? dispatch_epi<true>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch, f16, out_scale)
+                : dispatch_epi<false>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, epi, status, scratch, f16, out_scale);
 }
 
 }  // namespace nnc

@@ -215,7 +215,7 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
         } else {
             NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
                                                    c.n_kv_heads, c.max_seq, m->d_len, nullptr));
-            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, c.n_q_heads, c.n_kv_heads, c.max_seq, m->d_len));
+            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, false, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len));
         }
         NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
         NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
@@ -726,14 +726,15 @@ int nnc_op_attn_decode(const float *q, const void *kcache, const void *vcache, f
 }
 
 int nnc_op_attn_prefill(const float *qkv, const void *kcache, const void *vcache, void *out, void *out_lo, int32_t batch,
-                        int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, const int32_t *n_past_dev,
-                        void *cuda_stream) {
-    if (!qkv || !kcache || !vcache || !out || !n_past_dev) return NNC_ERR_INVALID_ARG;
-    if (batch <= 0 || T <= 0 || n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % n_kv_heads || max_seq < T) return NNC_ERR_INVALID_ARG;
+                        int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_past, void *cuda_stream) {
+    if (!qkv || !kcache || !vcache || !out) return NNC_ERR_INVALID_ARG;
+    if (batch <= 0 || T <= 0 || n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % n_kv_heads || n_past < 0) return NNC_ERR_INVALID_ARG;
+    if ((long)n_past + T > max_seq) return NNC_ERR_CAPACITY;
     LaunchCtx lc;
     if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
-    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, (const bf16 *)kcache, (const bf16 *)vcache, (bf16 *)out,
-                                        (bf16 *)out_lo, n_q_heads, n_kv_heads, max_seq, n_past_dev);
+    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, (const bf16 *)kcache, (const bf16 *)vcache, out, out_lo, false,
+                                        n_q_heads, n_kv_heads, max_seq, n_past);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 

@@ -84,8 +84,9 @@ cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
                                        const int32_t *d_len, bf16 *q_bf16_out);
+// out_f16: `out` receives one fp16 matrix (saturating) instead of a bf16 value (+ residual in out_lo)
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
-                                int H, float eps, int first, int step);
+                                int H, float eps, int first, int step, bool out_f16 = false);
 cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n);
 cudaError_t launch_add_len(const LaunchCtx &lc, int32_t *d_len, int delta);
 
@@ -105,9 +106,11 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
                                float *out_f32, bf16 *out_bf16, bf16 *out_bf16_lo, int out_row_stride, float *part,
                                uint32_t *tickets, const int32_t *d_len, int len_add, int batch, int nq, int nkv,
                                int max_seq, int n_splits, const AttnFused *fused);
+// prompt-phase causal attention on the tcgen05 path (attn_prefill_tc.cu); out: bf16 value (+ residual in out_lo, nullable)
+// or, with out_fp16, one fp16 matrix.  n_past (cached positions before this call) is a host value: it sizes the tensor maps.
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
-                                const bf16 *vcache, bf16 *out, bf16 *out_lo, int nq, int nkv, int max_seq,
-                                const int32_t *d_len);
+                                const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
+                                int n_past);
 
 // ---- GEMM (gemm_tc.cu) --------------------------------------------------------------------------------
 enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwigluBf16 = 3 };
@@ -124,12 +127,18 @@ struct GemmScratch {
 };
 constexpr size_t kGemmPartBytes = 48u << 20;
 constexpr int kGemmTickets = 4096;
+// f16: X and W hold fp16 (single term, T > 128 only) and the SwiGLU epilogue writes fp16; out_scale (nullable): DEVICE
+// scalar multiplied into the accumulators, undoing the power-of-two scale of an fp16 weight copy.
 cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T,
-                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch = nullptr);
+                        int N, int K, int ldy, int epi, int *status, const GemmScratch *scratch = nullptr, bool f16 = false,
+                        const float *out_scale = nullptr);
 
 // ---- repack (repack.cu) -------------------------------------------------------------------------------
 // dst rows [row0, row0 + rows) <- src rows [0, rows), row length K (plain row copy into a taller matrix)
 cudaError_t launch_copy_rows(const LaunchCtx &lc, const bf16 *src, bf16 *dst, int rows, int K, int dst_row0,
                              int dst_row_step, int src_row0, int src_row_step);
+
+// fp16 copy of a bf16 matrix scaled by a power of two (see repack.cu); scales: DEVICE float[2] <- {2^e, 2^-e}
+cudaError_t launch_to_f16_scaled(const LaunchCtx &lc, const bf16 *src, void *dst, size_t n, float *scales, uint32_t *max_bits);
 
 }  // namespace nnc

@@ -1,6 +1,14 @@
 // One-time weight repack (and its inverse, for tests): strided row copies between bf16 matrices whose rows
 // have the same length.  Concatenating Wq|Wk|Wv and interleaving gate/up rows are both instances of
 // "destination row d0 + i*ds <- source row s0 + i*ss".  Pure bit moves, 16 bytes per thread, HBM-bound.
+//
+// Also here: the fp16 copy of a bf16 matrix that the prompt-phase GEMMs multiply with fp16 activations.  fp16 has more
+// mantissa bits than bf16 but a narrow exponent range, so the copy holds W * 2^e with e chosen per matrix such that
+// the largest magnitude lands in [2^14, 2^15): every weight down to 2^-38 of the largest one converts exactly (the 8
+// significant bits of a bf16 value fit, and the scaling is a power of two); smaller ones round on the fp16 subnormal
+// grid, an error below 2^-39 of the largest weight.  The GEMM epilogue multiplies by 2^-e.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "nnc_internal.h"
 
@@ -18,7 +26,75 @@ __global__ void copy_rows_kernel(const uint4 *__restrict__ src, uint4 *__restric
     }
 }
 
+// max |w| over a bf16 matrix as fp32 bits (non-negative floats order like their bit patterns); NaNs are skipped
+__global__ void absmax_bits_kernel(const uint4 *__restrict__ src, size_t n_chunks, uint32_t *__restrict__ max_bits) {
+    uint32_t m = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_chunks; i += (size_t)gridDim.x * blockDim.x) {
+        const uint4 v = src[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t a = (w[k] << 16) & 0x7fffffffu, b = w[k] & 0x7fff0000u;
+            if (a <= 0x7f800000u && a > m) m = a;
+            if (b <= 0x7f800000u && b > m) m = b;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m) atomicMax(max_bits, m);
+}
+
+// scales[0] = 2^e, scales[1] = 2^-e with 2^14 <= max * 2^e < 2^15 (e = 0 for an all-zero or non-finite maximum)
+__global__ void f16_scale_kernel(const uint32_t *__restrict__ max_bits, float *__restrict__ scales) {
+    const uint32_t b = *max_bits;
+    int e = 0;
+    if (b != 0 && b < 0x7f800000u) {
+        int ex = (int)(b >> 23) - 127;           // floor(log2(max)) for normal values
+        if ((b >> 23) == 0) ex = -127;           // bf16 subnormals: treat as the smallest normal binade
+        e = 14 - ex;
+        if (e > 120) e = 120;
+        if (e < -120) e = -120;
+    }
+    scales[0] = exp2f((float)e);
+    scales[1] = exp2f((float)-e);
+}
+
+__global__ void to_f16_scaled_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n_chunks,
+                                     const float *__restrict__ scales) {
+    const float sc = scales[0];
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_chunks; i += (size_t)gridDim.x * blockDim.x) {
+        const uint4 v = src[i];
+        uint4 o;
+        o.x = pack_f16x2_sat(bf16_lo(v.x) * sc, bf16_hi(v.x) * sc);
+        o.y = pack_f16x2_sat(bf16_lo(v.y) * sc, bf16_hi(v.y) * sc);
+        o.z = pack_f16x2_sat(bf16_lo(v.z) * sc, bf16_hi(v.z) * sc);
+        o.w = pack_f16x2_sat(bf16_lo(v.w) * sc, bf16_hi(v.w) * sc);
+        dst[i] = o;
+    }
+}
+
 }  // namespace
+
+// dst (fp16 bits) = src (bf16) * 2^e; scales: DEVICE float[2] receiving {2^e, 2^-e}; max_bits: DEVICE scratch word.
+// Stream-ordered, no host synchronisation.
+cudaError_t launch_to_f16_scaled(const LaunchCtx &lc, const bf16 *src, void *dst, size_t n, float *scales, uint32_t *max_bits) {
+    if (n % 8) return cudaErrorInvalidValue;
+    const size_t chunks = n / 8;
+    size_t blocks = (chunks + 255) / 256;
+    const size_t cap = (size_t)lc.sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks == 0) return cudaSuccess;
+    LaunchCtx plain = lc;
+    plain.pdl = false;
+    cudaError_t e = cudaMemsetAsync(max_bits, 0, 4, lc.stream);
+    if (e != cudaSuccess) return e;
+    e = launch(plain, absmax_bits_kernel, dim3((unsigned)blocks), dim3(256), reinterpret_cast<const uint4 *>(src), chunks, max_bits);
+    if (e != cudaSuccess) return e;
+    e = launch(plain, f16_scale_kernel, dim3(1), dim3(1), (const uint32_t *)max_bits, scales);
+    if (e != cudaSuccess) return e;
+    return launch(plain, to_f16_scaled_kernel, dim3((unsigned)blocks), dim3(256), reinterpret_cast<const uint4 *>(src),
+                  reinterpret_cast<uint4 *>(dst), chunks, (const float *)scales);
+}
 
 cudaError_t launch_copy_rows(const LaunchCtx &lc, const bf16 *src, bf16 *dst, int rows, int K, int dst_row0,
                              int dst_row_step, int src_row0, int src_row_step) {

@@ -176,15 +176,24 @@ def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
     assert torch.allclose(Yb.float(), ref.float(), rtol=2e-2, atol=2e-2)
 
 
-@pytest.mark.parametrize("batch,T,nq,nkv,n_past", [(1, 19, 2, 1, 0), (2, 130, 4, 2, 7), (1, 300, 8, 2, 0), (1, 64, 16, 8, 200)])
-def test_attn_prefill_against_oracle(nnc, oracle_mod, batch, T, nq, nkv, n_past):
+@pytest.mark.parametrize("batch,T,nq,nkv,n_past,growth", [
+    (1, 19, 2, 1, 0, 0.0), (2, 130, 4, 2, 7, 0.0), (1, 300, 8, 2, 0, 0.0), (1, 64, 16, 8, 200, 0.0),
+    (1, 128, 1, 1, 0, 0.0), (1, 129, 2, 2, 127, 0.0),            # exactly one tile; one row past a tile boundary
+    (1, 2048, 4, 1, 100, 0.0),                                    # the prompt length of the batched workload, with a past
+    (1, 700, 2, 1, 60, 0.15), (1, 400, 2, 2, 0, 1.0)])            # keys that grow along the sequence: the running maximum moves
+def test_attn_prefill_against_oracle(nnc, oracle_mod, batch, T, nq, nkv, n_past, growth):
     """Causal prompt-phase attention: query s sees cache positions 0 .. n_past + s.  Rows are checked against the
-    oracle's single-query attention over the matching cache prefix (sampled rows, all heads of those rows)."""
+    oracle's single-query attention over the matching cache prefix (sampled rows, all heads of those rows).  With
+    `growth` the keys of each further block of 128 positions are larger, so a later tile's score maximum exceeds the
+    running one by a little (0.15) or by far (1.0) and the accumulator is rescaled on the way."""
     max_seq = n_past + T + 5
     heads = nq + 2 * nkv
     qkv = synth.normal(9, 1, (batch * T, heads * 128), 1.0, torch.float32, "cuda")
     kc = synth.normal(9, 2, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
     vc = synth.normal(9, 3, (batch, nkv, max_seq, 128), 1.0, torch.bfloat16, "cuda")
+    if growth:
+        blk = (torch.arange(max_seq, device="cuda") // 128).float()
+        kc = (kc.float() * (1.0 + growth * blk).view(1, 1, -1, 1)).to(torch.bfloat16).contiguous()
     kc[:, :, n_past + T:] = float("nan"); vc[:, :, n_past + T:] = float("nan")   # never to be read into a result
     out, out_lo = nnc.op_attn_prefill(qkv, kc, vc, T, nq, n_past)
     torch.cuda.synchronize()
@@ -193,7 +202,7 @@ def test_attn_prefill_against_oracle(nnc, oracle_mod, batch, T, nq, nkv, n_past)
     G = nq // nkv
     qc, kcc, vcc = qkv.cpu().view(batch, T, heads, 128), kc.cpu(), vc.cpu()
     for b in range(batch):
-        for s in sorted(set([0, 1, T // 2, T - 1, min(T - 1, 127), min(T - 1, 128)])):
+        for s in sorted(set([0, 1, T // 2, T - 1, min(T - 1, 127), min(T - 1, 128), min(T - 1, 255), (2 * T) // 3])):
             n = n_past + s + 1
             for h in range(nq):
                 want = oracle_mod.attend(qc[b, s, h].contiguous(), kcc[b, h // G, :n].contiguous(), vcc[b, h // G, :n].contiguous())
