@@ -10,8 +10,11 @@ step, or one prompt-phase call.  Prints ONE JSON line (rank 0).  Inputs are seed
   value      device-timed throughput, inputs resident in HBM (CUDA events on the launching stream)
   e2e        the same metric through the *_host entry points: host->device copy of the tokens and
              device->host copy of the logits inside the timed region, one synchronisation per step
-  roofline   the dominant kernel timed alone over operands larger than L2, against the measured peak
+  roofline   the dominant kernel timed alone over operands larger than L2, against the measured peak: launched
+             back to back the way the step launches it (`frac`), and one launch at a time (`isolated_frac`)
   step_roofline  algorithmic bytes (or FLOPs) of a whole step over the step time
+  prefill    (default workload only) the prompt-phase half of the metric: one call of 4 x 2048 tokens on the same
+             model shape, tokens/s and model FLOPs over the measured bf16 tensor-core peak
   cpu_baseline   the CPU oracle, as it stands, on the host cores, on a bounded sample of the workload
 
 With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent replica: the forward
@@ -58,6 +61,25 @@ def load_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
                     bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def measured_traffic(key: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel from the profiler capture
+    recorded in profiles/dram_traffic.json -- or None when there is no capture for `key` or the kernel's source file
+    has changed since the capture was taken (the record holds the file's SHA-1 at that time)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f).get(key)
+        if not rec:
+            return None
+        with open(os.path.join(ROOT, rec["source"]), "rb") as f:
+            if hashlib.sha1(f.read()).hexdigest() != rec["source_sha1"]:
+                return None
+        return float(rec["bytes_per_launch"])
+    except (OSError, ValueError, KeyError):
+        return None
 
 
 class ClockSampler:
@@ -161,11 +183,12 @@ def whole_job_throughput(ms_local: float, steps: int, units_per_step: int, world
     return ms, world * steps * units_per_step / (ms * 1e-3)
 
 
-def build_model(wl, max_tokens=None):
+def build_model(wl, max_tokens=None, w=None):
     from paper_2512_21571_b200 import binding
     shape = synth.SHAPES[wl["shape"]]
     seed = wl["seed"]
-    w = synth.make_weights(shape, seed, device="cuda")
+    if w is None:
+        w = synth.make_weights(shape, seed, device="cuda")
     if wl["kind"] == "decode":
         max_seq = wl["ctx"] + wl["pass_steps"]
         mt = max(wl["batch"], 1)
@@ -194,6 +217,21 @@ def prefill_flops(shape, batch, T):
     attn = 2.0 * 2.0 * batch * shape.n_layers * shape.n_q_heads * shape.head_dim * (T * (T + 1) / 2)
     head = 2.0 * batch * shape.vocab * shape.hidden  # last position only
     return proj, attn, head
+
+
+def prefill_roofline(shape, wl, ms_per_call, peaks):
+    """Model FLOPs of one prompt-phase call over its time, against the measured bf16 tensor-core peaks; `issued` adds
+    the second bf16 term of the operands that are fed as value + residual (QKV input, Q and P inside attention)."""
+    proj, attn, head = prefill_flops(shape, wl["batch"], wl["tokens"])
+    total = proj + attn + head
+    qkv = 2.0 * wl["batch"] * wl["tokens"] * shape.n_layers * (shape.q_dim + 2 * shape.kv_dim) * shape.hidden
+    issued = total + qkv + attn
+    ach = total / (ms_per_call * 1e-3) / 1e12
+    return {"bound": "tensor", "flops_per_step": total, "projection_flops": proj, "attention_flops": attn,
+            "achieved": round(ach, 1), "unit": "TFLOP/s (model FLOPs)",
+            "peak": peaks["bf16_tflops"], "frac": round(ach / peaks["bf16_tflops"], 4), "peak_source": peaks["source"] + " (burst)",
+            "frac_of_sustained": round(ach / peaks["bf16_tflops_sustained"], 4), "frac_of_nominal_2250": round(ach / 2250.0, 4),
+            "issued_tflops": round(issued / (ms_per_call * 1e-3) / 1e12, 1)}
 
 
 def time_decode(m, shape, wl, steps, warmup, world):
@@ -303,67 +341,86 @@ def kernel_roofline_gemv(shape, peaks, w):
     x = synth.normal(9, 1, (H,), 1.0, torch.float32, "cuda")
     gain = torch.ones(H, dtype=torch.bfloat16, device="cuda")
     y = torch.empty(I, dtype=torch.float32, device="cuda")
-    reps = 3 if mats[0].numel() * 2 * n_mats > 4 * L2_BYTES else 0
+    reps = 3 if mats[0].numel() * 2 * n_mats > 4 * L2_BYTES else 1
     for W in mats[:3]:
         binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=True)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n = 0
     e0.record()
-    for _ in range(max(reps, 1)):
+    for _ in range(reps):
         for W in mats:
             binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=True)   # launched as inside the decode graph
             n += 1
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / n
+    # one launch at a time: plain stream order, an event pair around every launch, so no launch hides its start-up
+    # under its predecessor's tail
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in mats]
+    for (a, b), W in zip(pairs, mats):
+        a.record()
+        binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=False)
+        b.record()
+    torch.cuda.synchronize()
+    iso = sorted(a.elapsed_time(b) * 1e3 for a, b in pairs)
+    us_iso = iso[len(iso) // 2]
     nbytes = 2 * I * H * 2
     ach = nbytes / (us * 1e-6) / 1e9
+    ach_iso = nbytes / (us_iso * 1e-6) / 1e9
     return {"bound": "hbm", "kernel": "gemv_stream_kernel<SwiGLU, norm prologue>", "shape": [2 * I, H],
             "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
             "peak_source": peaks["source"], "bytes_per_launch": nbytes, "us_per_launch": round(us, 2),
-            "launches_timed": n,
-            # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/gemv_stream_kernel_gateup_qwen3-8b.md);
-            # valid for the 24576 x 4096 shape only
-            "traffic": 205.3e6 if (2 * I, H) == (24576, 4096) else None}
+            "launches_timed": n, "how": "back-to-back launches with programmatic stream serialization, as in the decode graph",
+            "isolated_us_per_launch": round(us_iso, 2), "isolated_achieved": round(ach_iso, 1),
+            "isolated_frac": round(ach_iso / peaks["hbm_gbs"], 4),
+            "traffic": measured_traffic("gemv_stream_kernel<SwiGLU>:%dx%d" % (2 * I, H))}
 
 
 def kernel_roofline_gemm(shape, peaks, T):
-    """The dominant prompt-phase kernel -- the tcgen05 GEMM on the gate/up shape -- timed alone."""
+    """The dominant prompt-phase kernel -- the tcgen05 GEMM on the gate/up shape with the SwiGLU epilogue -- timed
+    alone in the form the prompt phase uses (one fp16 term, scaled fp16 weight copy).  `achieved` counts MODEL FLOPs,
+    2 * T * 2I * H per launch; the two-bf16-term form of the same product is reported beside it."""
     from paper_2512_21571_b200 import binding
     H, I = shape.hidden, shape.intermediate
     X = synth.normal(9, 1, (T, H), 1.0, torch.bfloat16, "cuda")
     X_lo = synth.normal(9, 2, (T, H), 0.004, torch.bfloat16, "cuda")
     W = synth.normal(9, 3, (2 * I, H), 0.02, torch.bfloat16, "cuda")
+    X16 = X.to(torch.float16)
+    W16, scales = binding.op_to_f16_scaled(W)
+    model_flops = 2.0 * T * 2 * I * H
+    runs = {"f16": lambda: binding.op_gemm_swiglu_f16(X16, W16, out_scale=scales[1:]),
+            "bf16_two_terms": lambda: binding.op_gemm_swiglu(X, W, X_lo=X_lo)}
+    if T <= 128:
+        runs.pop("f16")
     out = {}
-    for name, lo in (("split", X_lo), ("single", None)):
+    for name, fn in runs.items():
         for _ in range(3):
-            binding.op_gemm_swiglu(X, W, X_lo=lo)
+            fn()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n = 10
         e0.record()
         for _ in range(n):
-            binding.op_gemm_swiglu(X, W, X_lo=lo)
+            fn()
         e1.record()
         torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) * 1e3 / n
-        mma_flops = 2.0 * T * 2 * I * H * (2 if lo is not None else 1)
-        out[name] = (us, mma_flops)
+        out[name] = e0.elapsed_time(e1) * 1e3 / n
     assert binding.op_status() == 0
-    us, fl = out["split"]
-    ach = fl / (us * 1e-6) / 1e12
-    us1, fl1 = out["single"]
-    return {"bound": "tensor", "kernel": "gemm_tc_kernel<SwiGLU, value+residual activations>", "shape": [T, 2 * I, H],
-            "achieved": round(ach, 1), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-            "frac": round(ach / peaks["bf16_tflops"], 4), "peak_source": peaks["source"],
-            "flops_per_launch": fl, "us_per_launch": round(us, 1), "launches_timed": 10, "traffic": None,
-            "single_term": {"achieved": round(fl1 / (us1 * 1e-6) / 1e12, 1), "us_per_launch": round(us1, 1)}}
-
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the flash-decode from one ncu capture of this very
-# configuration (profiles/attn_decode_kernel_qwen3-8b_b32_ctx8192.md); to be set back to None when the kernel changes
-ATTN_DRAM_TRAFFIC = {(32, 8, 32, 8192): 1.0831e9}
+    head = "f16" if "f16" in out else "bf16_two_terms"
+    us = out[head]
+    ach = model_flops / (us * 1e-6) / 1e12
+    res = {"bound": "tensor", "kernel": "gemm_tc_kernel<SwiGLU, %s>" % ("one fp16 term" if head == "f16" else "two bf16 terms"),
+           "shape": [T, 2 * I, H], "achieved": round(ach, 1), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+           "frac": round(ach / peaks["bf16_tflops"], 4), "peak_source": peaks["source"] + " (burst; fp16 and bf16 share the rate)",
+           "frac_of_sustained": round(ach / peaks["bf16_tflops_sustained"], 4),
+           "flops_per_launch": model_flops, "us_per_launch": round(us, 1), "launches_timed": 10,
+           "traffic": measured_traffic("gemm_tc_kernel<SwiGLU,f16>:%dx%dx%d" % (T, 2 * I, H)) if head == "f16" else None}
+    if "bf16_two_terms" in out and head == "f16":
+        us2 = out["bf16_two_terms"]
+        res["bf16_two_terms"] = {"us_per_launch": round(us2, 1), "model_tflops": round(model_flops / (us2 * 1e-6) / 1e12, 1),
+                                 "issued_tflops": round(2 * model_flops / (us2 * 1e-6) / 1e12, 1)}
+    return res
 
 
 def kernel_roofline_attn(shape, peaks, batch, ctx):
@@ -393,7 +450,7 @@ def kernel_roofline_attn(shape, peaks, batch, ctx):
     return {"bound": "hbm", "kernel": "attn_decode_kernel<G=%d>" % (nq // nkv), "shape": [batch, nkv, ctx, 128],
             "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
             "peak_source": peaks["source"], "bytes_per_launch": int(nbytes), "us_per_launch": round(us, 2),
-            "launches_timed": n, "traffic": ATTN_DRAM_TRAFFIC.get((nq, nkv, batch, ctx))}
+            "launches_timed": n, "traffic": measured_traffic("attn_decode_kernel<G=%d>:b%d_ctx%d" % (nq // nkv, batch, ctx))}
 
 
 # ---- the CPU oracle leg (reported baseline; the only place the product's bench touches oracle/) ------------
@@ -557,16 +614,13 @@ def main():
         ms, value = whole_job_throughput(ms, steps, units_per_step, world)
         ms_e, _, _, h2d, d2h = time_prefill(m, shape, wl, steps, 1, world, host=True)
         ms_e, e2e_value = whole_job_throughput(ms_e, steps, units_per_step, world)
-        proj, attn, head = prefill_flops(shape, wl["batch"], wl["tokens"])
-        ach = (proj + attn + head) / (ms / steps * 1e-3) / 1e12
-        step_roof = {"bound": "tensor", "flops_per_step": proj + attn + head, "projection_flops": proj,
-                     "achieved": round(ach, 1), "unit": "TFLOP/s (model FLOPs; the value+residual activation feed doubles the tensor-core work)",
-                     "peak": peaks["bf16_tflops_sustained"], "frac": round(ach / peaks["bf16_tflops_sustained"], 4),
-                     "peak_source": peaks["source"] + " (sustained)", "frac_of_nominal_2250": round(ach / 2250.0, 4)}
+        step_roof = prefill_roofline(shape, wl, ms / steps, peaks)
 
     line = {"metric": metric_name(wl), "value": round(value, 2), "unit": "tokens/s", "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": round(ms / steps, 4), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "dtype_detail": "bf16 weights and KV cache, fp32 activations and accumulation",
+            "vs_baseline": None, "dtype": "bf16",
+            "dtype_detail": "bf16 weights and KV cache, fp32 residual stream and accumulation; tensor-core operands: two bf16 "
+                            "terms, or one fp16 term with exact fp16 weight copies (prompt phase: O, gate/up, down)",
             "data": "synthetic",
             "config": config_of(wl), "clocks": clocks,
             "e2e": {"value": round(e2e_value, 2), "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -583,6 +637,26 @@ def main():
             T = wl["batch"] * wl.get("tokens", 1)
             line["roofline"] = kernel_roofline_gemm(shape, peaks, max(T, 32))
     m.close()
+    del m
+    if wl is WORKLOADS[DEFAULT_WORKLOAD] and not args.no_extras:
+        # the prompt-phase half of the metric, same model shape and weights: one call of 4 x 2048 tokens
+        pwl = WORKLOADS["qwen3-8b-prefill-4x2048"]
+        torch.cuda.empty_cache()
+        pm, _, _ = build_model(pwl, w=w)
+        p_steps = 3
+        pms, p_launches, p_clocks, _, _ = time_prefill(pm, shape, pwl, p_steps, 3, world)
+        pms, p_value = whole_job_throughput(pms, p_steps, pwl["batch"] * pwl["tokens"], world)
+        pms_e, _, _, ph2d, pd2h = time_prefill(pm, shape, pwl, p_steps, 1, world, host=True)
+        pms_e, p_e2e = whole_job_throughput(pms_e, p_steps, pwl["batch"] * pwl["tokens"], world)
+        pm.close()
+        del pm
+        line["prefill"] = {"metric": metric_name(pwl), "value": round(p_value, 1), "unit": "tokens/s", "steps": p_steps, "warmup": 3,
+                           "ms_per_step": round(pms / p_steps, 3), "config": config_of(pwl), "clocks": p_clocks,
+                           "e2e": {"value": round(p_e2e, 1), "unit": "tokens/s", "h2d_bytes_per_step": ph2d,
+                                   "d2h_bytes_per_step": pd2h},
+                           "gpu_launches": int(p_launches), "step_roofline": prefill_roofline(shape, pwl, pms / p_steps, peaks)}
+        if rank == 0:
+            line["prefill"]["roofline"] = kernel_roofline_gemm(shape, peaks, pwl["batch"] * pwl["tokens"])
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, desc = oracle_leg(wl, shape, w, 12, 1)
         line["cpu_baseline"] = dict(desc, value=round(v, 4), unit="tokens/s")

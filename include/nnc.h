@@ -56,11 +56,26 @@ typedef struct {
     int32_t tie_embeddings; /* 1: the lm_head is the embedding matrix */
     float rms_eps;          /* 1e-6 for Qwen3 */
     float rope_theta;       /* 1e6 for Qwen3 */
-    int32_t fast_bf16_activations; /* tensor-core path only (prompt phase, batched decode).  0 (default): each
-                             * activation operand is fed as two bf16 terms, value + rounding residual, i.e. ~16
-                             * mantissa bits, which keeps deep models inside the parity tolerance at twice the
-                             * tensor-core work.  1: one bf16 term (half the tensor-core work; rounding error of
-                             * 2^-9 per operand accumulates to a few percent over ~30 layers). */
+    int32_t tc_operands;    /* operand feed of the tensor-core path (prompt phase, batched decode).  The residual stream
+                             * stays fp32 everywhere; this only says how an activation matrix enters a tcgen05.mma.
+                             * 0 (default): calls with more than 128 tokens multiply the attention output, the MLP input and
+                             *    the SwiGLU output as ONE fp16 term with fp16 copies of Wo, Wgate/up and Wdown (made at
+                             *    create time when max_tokens > 128; scaled by a power of two per matrix, exact for bf16
+                             *    weights), and the QKV input -- the operand deep models are sensitive to -- as TWO bf16
+                             *    terms (value + rounding residual, ~16 mantissa bits).  Calls with at most 128 tokens use
+                             *    two bf16 terms throughout (they are bound by streaming the weights, not by the MMAs).
+                             * 1: two bf16 terms throughout, no fp16 weight copies (smaller workspace, ~1.8x the tensor work
+                             *    of mode 0 in the prompt phase).
+                             * 2: one bf16 term throughout (half the tensor work of mode 1; 2^-9 per operand accumulates to
+                             *    a few percent of hidden-state error over ~30 layers, outside the parity tolerance). */
+    int32_t weight_format;  /* 0 (default): bf16 weights.  1: the second weight precision (the paper evaluates two, Section
+                             * 4.1) -- weight-only FP8: at create time every matrix that is multiplied (QKV, O, gate/up,
+                             * down, lm_head; a tied embedding is that same matrix) is quantised row by row to E4M3 codes
+                             * times a power-of-two scale 2^e per output row (e the smallest integer with max|w| <= 448 *
+                             * 2^e, round to nearest even, saturating), and the bf16 copy in the workspace is replaced by
+                             * the dequantised values (exact in bf16).  Batch-1 decode streams the codes (half the bytes per
+                             * step); the tensor-core paths multiply the dequantised bf16 matrices, so every path computes
+                             * the same model: the forward pass on the dequantised weights. */
     int32_t serial_launches; /* 0 (default): kernels are launched with programmatic stream serialization, so a
                              * kernel's set-up and weight prefetch overlap its predecessor's tail.  1: plain stream
                              * order (for debugging and for timing the overlap's worth). */
@@ -146,7 +161,7 @@ int nnc_layer_decode(nnc_model *model, int32_t layer, const float *x_in, float *
 
 /* Write the ORIGINAL (caller-layout) matrix back from the repacked store: which = 0 wq, 1 wk, 2 wv, 3 wo,
  * 4 w_gate, 5 w_up, 6 w_down; out DEVICE bf16 of that matrix's shape.  Lets a test check that the repack
- * loses nothing. */
+ * loses nothing (with weight_format 1 the store holds the dequantised values, and those are what comes back). */
 int nnc_unrepack(nnc_model *model, int32_t layer, int32_t which, void *out);
 
 /* Reads (and clears) the device status word; synchronises the stream.  0 = no kernel gave up on a wait. */
@@ -183,6 +198,19 @@ int nnc_op_gemm_swiglu(const void *X, const void *X_lo, const void *W, void *Y, 
  * must not overlap on the device.  With T > 128 it behaves as nnc_op_gemm. */
 int nnc_op_gemm_splitk(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
                        int32_t out_f32, int32_t accumulate, void *scratch, size_t scratch_bytes, void *cuda_stream);
+/* The fp16 forms used by the prompt phase: X fp16 [T][n_in] (T > 128), W fp16 [n_out][n_in], one term.  out_scale: NULL
+ * or a DEVICE float multiplied into every accumulator before the epilogue (undoes the scale of an fp16 weight copy).
+ * nnc_op_gemm_f16: Y fp32 [T][n_out], Y += product when accumulate != 0.  nnc_op_gemm_swiglu_f16: W rows interleaved
+ * gate/up, Y fp16 [T][n_out/2] (values beyond +-65504 saturate). */
+int nnc_op_gemm_f16(const void *X, const void *W, float *Y, int32_t T, int32_t n_out, int32_t n_in, int32_t accumulate,
+                    const float *out_scale, void *cuda_stream);
+int nnc_op_gemm_swiglu_f16(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                           const float *out_scale, void *cuda_stream);
+/* dst (fp16) = src (bf16) * 2^e, n elements (a multiple of 8), with e chosen so that the largest magnitude lands in
+ * [2^14, 2^15): exact for every element down to 2^-32 of the largest (smaller ones round with an error below 2^-39 of the largest).  scales: DEVICE float[2] receiving {2^e, 2^-e};
+ * scratch_word: DEVICE uint32 used during the call. */
+int nnc_op_to_f16_scaled(const void *src, void *dst, size_t n, float *scales, uint32_t *scratch_word, void *cuda_stream);
+
 /* Status word of the nnc_op_* tensor-core kernels (0 = no bounded wait ran out); synchronises the device and
  * clears the word.  status_out is a HOST pointer. */
 int nnc_op_status(int32_t *status_out);
@@ -196,6 +224,16 @@ int nnc_op_status(int32_t *status_out);
 #define NNC_GEMV_CHAINED 0x100
 int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t n_in, const void *gain,
                 float eps, int32_t mode, void *cuda_stream);
+
+/* FP8 E4M3 row quantisation (nnc_config::weight_format 1): W bf16 [n_out][n_in] -> codes uint8 [n_out][n_in] and
+ * scales fp32 [n_out] (= 2^e per row); dequant: NULL, or bf16 [n_out][n_in] receiving code * 2^e (may be W itself).
+ * n_in a multiple of 8. */
+int nnc_op_quantise_rows_e4m3(const void *W, void *codes, float *scales, void *dequant, int32_t n_out, int32_t n_in,
+                              void *cuda_stream);
+/* nnc_op_gemv on FP8 weights: y = diag(scales) * codes * x with the same modes, gain and chaining flag; n_in a multiple
+ * of 16 (up to 16384; 8192 with mode 2). */
+int nnc_op_gemv_fp8(const void *codes, const float *scales, const float *x, float *y, int32_t n_out, int32_t n_in,
+                    const void *gain, float eps, int32_t mode, void *cuda_stream);
 
 /* Split-K flash-decode for one query token per sequence over a contiguous cache.
  *   q fp32 [batch][n_q_heads][128] (already normalised and rotated);  kcache, vcache bf16

@@ -24,8 +24,8 @@ lib = C.CDLL(LIB_PATH)
 class nnc_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "intermediate",
                                          "vocab", "max_seq", "max_batch", "max_tokens", "tie_embeddings")] + \
-               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("fast_bf16_activations", C.c_int32),
-                ("serial_launches", C.c_int32)]
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("tc_operands", C.c_int32),
+                ("weight_format", C.c_int32), ("serial_launches", C.c_int32)]
 
 
 LAYER_FIELDS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "g_in", "g_post", "g_q", "g_k")
@@ -66,9 +66,17 @@ EXPORTS = {
                                      C.c_int32, C.c_void_p]),
     "nnc_op_gemm_splitk": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "nnc_op_gemm_f16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                  C.c_void_p]),
+    "nnc_op_gemm_swiglu_f16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                         C.c_void_p]),
+    "nnc_op_to_f16_scaled": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]),
     "nnc_op_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "nnc_op_gemv": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_float, C.c_int32,
                               C.c_void_p]),
+    "nnc_op_quantise_rows_e4m3": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "nnc_op_gemv_fp8": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_float,
+                                  C.c_int32, C.c_void_p]),
     "nnc_attn_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
     "nnc_op_attn_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
@@ -101,13 +109,14 @@ class Model:
     """nnc_model_create / nnc_prefill / nnc_decode_step and the auxiliary calls, one method per C function."""
 
     def __init__(self, shape, weights: dict, max_seq: int, max_batch: int = 1, max_tokens: Optional[int] = None,
-                 fast_bf16_activations: bool = False, serial_launches: bool = False):
+                 tc_operands: int = 0, serial_launches: bool = False,
+                 weight_format: int = 0):
         self.shape = shape
         self.cfg = nnc_config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                               shape.intermediate, shape.vocab, max_seq, max_batch,
                               max_tokens if max_tokens is not None else max(max_batch, 1),
                               int(shape.tie_embeddings), shape.rms_eps, shape.rope_theta,
-                              int(fast_bf16_activations), int(serial_launches))
+                              int(tc_operands), int(weight_format), int(serial_launches))
         self.handle = C.c_void_p()
         nbytes = lib.nnc_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
@@ -250,6 +259,37 @@ def op_gemm_swiglu(X: torch.Tensor, W: torch.Tensor, X_lo: Optional[torch.Tensor
     return (Y, Y_lo) if want_lo else Y
 
 
+def op_to_f16_scaled(W: torch.Tensor):
+    """nnc_op_to_f16_scaled: (fp16 copy of W * 2^e, scales tensor {2^e, 2^-e} on the device)."""
+    out = torch.empty(W.shape, dtype=torch.float16, device="cuda")
+    scales = torch.zeros(2, dtype=torch.float32, device="cuda")
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _ok(lib.nnc_op_to_f16_scaled(_dev(W, torch.bfloat16), out.data_ptr(), W.numel(), scales.data_ptr(), word.data_ptr(),
+                                 _stream_ptr()), "nnc_op_to_f16_scaled")
+    return out, scales
+
+
+def op_gemm_f16(X: torch.Tensor, W: torch.Tensor, out_scale: Optional[torch.Tensor] = None,
+                accumulate_into: Optional[torch.Tensor] = None):
+    T, K = X.shape
+    N = W.shape[0]
+    Y = accumulate_into if accumulate_into is not None else torch.empty(T, N, dtype=torch.float32, device="cuda")
+    _ok(lib.nnc_op_gemm_f16(_dev(X, torch.float16), _dev(W, torch.float16), _dev(Y, torch.float32), T, N, K,
+                            int(accumulate_into is not None), out_scale.data_ptr() if out_scale is not None else None,
+                            _stream_ptr()), "nnc_op_gemm_f16")
+    return Y
+
+
+def op_gemm_swiglu_f16(X: torch.Tensor, W: torch.Tensor, out_scale: Optional[torch.Tensor] = None):
+    T, K = X.shape
+    N = W.shape[0]
+    Y = torch.empty(T, N // 2, dtype=torch.float16, device="cuda")
+    _ok(lib.nnc_op_gemm_swiglu_f16(_dev(X, torch.float16), _dev(W, torch.float16), Y.data_ptr(), T, N, K,
+                                   out_scale.data_ptr() if out_scale is not None else None, _stream_ptr()),
+        "nnc_op_gemm_swiglu_f16")
+    return Y
+
+
 def op_status() -> int:
     st = C.c_int32(0)
     lib.nnc_op_status(C.byref(st))
@@ -267,6 +307,30 @@ def op_gemv(W: torch.Tensor, x: torch.Tensor, mode: int = 0, gain: Optional[torc
     _ok(lib.nnc_op_gemv(_dev(W, torch.bfloat16), _dev(x, torch.float32), _dev(y, torch.float32), N, K,
                         _dev(gain, torch.bfloat16) if gain is not None else None, eps,
                         mode | (GEMV_CHAINED if chained else 0), _stream_ptr()), "nnc_op_gemv")
+    return y
+
+
+def op_quantise_rows_e4m3(W: torch.Tensor, want_dequant: bool = True):
+    """nnc_op_quantise_rows_e4m3: (codes uint8, scales fp32 [n_out], dequantised bf16 or None)."""
+    n_out, n_in = W.shape
+    codes = torch.empty(n_out, n_in, dtype=torch.uint8, device="cuda")
+    scales = torch.empty(n_out, dtype=torch.float32, device="cuda")
+    dq = torch.empty_like(W) if want_dequant else None
+    _ok(lib.nnc_op_quantise_rows_e4m3(_dev(W, torch.bfloat16), codes.data_ptr(), scales.data_ptr(),
+                                      dq.data_ptr() if want_dequant else None, n_out, n_in, _stream_ptr()),
+        "nnc_op_quantise_rows_e4m3")
+    return codes, scales, dq
+
+
+def op_gemv_fp8(codes: torch.Tensor, scales: torch.Tensor, x: torch.Tensor, mode: int = 0,
+                gain: Optional[torch.Tensor] = None, eps: float = 1e-6, y: Optional[torch.Tensor] = None,
+                chained: bool = False):
+    N, K = codes.shape
+    if y is None:
+        y = torch.empty(N // 2 if (mode & 0xff) == 2 else N, dtype=torch.float32, device="cuda")
+    _ok(lib.nnc_op_gemv_fp8(_dev(codes, torch.uint8), _dev(scales, torch.float32), _dev(x, torch.float32),
+                            _dev(y, torch.float32), N, K, _dev(gain, torch.bfloat16) if gain is not None else None, eps,
+                            mode | (GEMV_CHAINED if chained else 0), _stream_ptr()), "nnc_op_gemv_fp8")
     return y
 
 

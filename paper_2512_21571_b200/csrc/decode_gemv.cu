@@ -238,9 +238,12 @@ cudaError_t launch_rows(const LaunchCtx &lc, const bf16 *W, const float *x, floa
 
 }  // namespace
 
-cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
+cudaError_t launch_gemv(const LaunchCtx &lc, const void *Wv, const float *wscale, const float *x, float *y, int n_out, int n_in,
                         const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr) {
-    if (gemv_stream_supported(n_out, n_in, mode)) return launch_gemv_stream(lc, W, x, y, n_out, n_in, gain, eps, mode, am, ctr);
+    if (wscale)   // FP8 codes: the streaming form only
+        return launch_gemv_stream(lc, Wv, wscale, 1, x, y, n_out, n_in, gain, eps, mode, am, ctr);
+    const bf16 *W = reinterpret_cast<const bf16 *>(Wv);
+    if (gemv_stream_supported(n_out, n_in, mode)) return launch_gemv_stream(lc, W, nullptr, 2, x, y, n_out, n_in, gain, eps, mode, am, ctr);
     if (n_in % 8 != 0 || n_in <= 0 || n_out <= 0 || (size_t)n_in * 4 > 200 * 1024) return cudaErrorInvalidValue;
     ArgmaxScratch a = am ? *am : ArgmaxScratch{nullptr, nullptr, nullptr, nullptr};
     const bool norm = gain != nullptr;

@@ -19,7 +19,12 @@
 //     free.  The ring takes more than half of an SM's shared memory on purpose: two of these CTAs can never share
 //     an SM, so each kernel's 148 CTAs land one per SM (with smaller rings the block scheduler was seen to stack
 //     two CTAs of one kernel on some SMs and leave others idle whenever the previous kernel still held space).
+// Second weight precision (the paper evaluates two, Section 4.1): the same kernel streams FP8 E4M3 codes with one
+// power-of-two scale per output row (half the bytes per step).  A 16-byte chunk then carries 16 weights; codes are
+// widened pairwise (cvt e4m3x2 -> f16x2 -> fp32) and multiplied in fp32; the row scale is applied to the finished
+// sum together with 1/rms.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word and drains.
+#include <cuda_fp16.h>
 #include <stdio.h>
 #include <stdlib.h>
 
@@ -87,12 +92,43 @@ __device__ __forceinline__ float dot_slice(const uint4 (&w)[J], const float (&xr
     return s;
 }
 
+// two E4M3 codes (low 16 bits of `pair`) -> two floats
+__device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t pair) {
+    uint32_t h2;
+    asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %1;\ncvt.rn.f16x2.e4m3x2 %0, lo;\n}" : "=r"(h2) : "r"(pair));
+    return __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+}
+
+// the same for 16-byte chunks of 16 E4M3 codes: xr holds the 16 matching activations
+template <int J>
+__device__ __forceinline__ float dot_slice_fp8(const uint4 (&w)[J], const float (&xr)[J][16]) {
+    float a[J][2];
+#pragma unroll
+    for (int i = 0; i < J; ++i) {
+        const uint32_t q[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+        a[i][0] = 0.f; a[i][1] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 lo = e4m3x2_to_float2(q[k]), hi = e4m3x2_to_float2(q[k] >> 16);
+            a[i][0] = fmaf(lo.x, xr[i][4 * k], a[i][0]);
+            a[i][1] = fmaf(lo.y, xr[i][4 * k + 1], a[i][1]);
+            a[i][0] = fmaf(hi.x, xr[i][4 * k + 2], a[i][0]);
+            a[i][1] = fmaf(hi.y, xr[i][4 * k + 3], a[i][1]);
+        }
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < J; ++i) s += a[i][0] + a[i][1];
+    return s;
+}
+
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
 
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
 struct StreamParams {
     const uint8_t *W;
+    const float *wscale;   // FP8 weights: one scale per output row (null for bf16 weights)
     const float *x;
     float *y;
     const bf16 *gain;
@@ -110,9 +146,11 @@ struct StreamParams {
     ArgmaxScratch am;
 };
 
-// J = 16-byte chunks per lane per row slice (kw <= J * 256).
-template <int J, int MODE, bool NORM>
+// J = 16-byte chunks per lane per row slice (kw <= J * 32 * CE elements).  WB = bytes per weight: 2 (bf16) or 1 (FP8
+// E4M3 codes with a scale per row); CE = weights per 16-byte chunk.
+template <int J, int MODE, bool NORM, int WB>
 __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
+    constexpr int CE = 16 / WB;
     NNC_TRACE_SCOPE(10 + MODE + 100 * (p.K / 1024));
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ __align__(8) uint64_t full[kMaxStages], empty[kMaxStages];
@@ -127,7 +165,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages;
-    const uint32_t row_bytes = (uint32_t)p.K * 2u;
+    const uint32_t row_bytes = (uint32_t)p.K * (uint32_t)WB;
     const uint32_t stage_bytes = (uint32_t)p.rps * row_bytes;
 
     if (threadIdx.x == 0) {
@@ -189,12 +227,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     const int ks = warp % ksplit, gi = warp / ksplit;
     const int rw = p.rps / gpi;   // rows this warp owns in each stage: gi, gi + gpi, ...
     // gains are weights: fetch them before waiting on the kernel that produces x
-    uint4 gr[NORM ? J : 1];
+    uint4 gr[NORM ? J : 1][CE / 8];
     if (NORM) {
 #pragma unroll
         for (int i = 0; i < J; ++i) {
             const int c = lane + 32 * i;
-            gr[i] = (c * 8 < p.kw) ? *reinterpret_cast<const uint4 *>(p.gain + (size_t)ks * p.kw + (size_t)c * 8) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int h = 0; h < CE / 8; ++h)
+                gr[i][h] = (c * CE < p.kw) ? *reinterpret_cast<const uint4 *>(p.gain + (size_t)ks * p.kw + (size_t)c * CE + 8 * h)
+                                           : make_uint4(0, 0, 0, 0);
         }
     }
     pdl_wait();
@@ -202,28 +243,33 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
 
     // this warp's activation slice, in registers.  With the norm prologue it holds x * gain; the scalar
     // 1/rms(x) is applied to the finished row sums at the fold, so nothing waits for the sum of squares.
-    float xr[J][8];
+    float xr[J][CE];
     float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < J; ++i) {
         const int c = lane + 32 * i;
-        if (c * 8 < p.kw) {
-            const float4 *xp = reinterpret_cast<const float4 *>(p.x + (size_t)ks * p.kw + (size_t)c * 8);
-            const float4 a = xp[0], b = xp[1];
-            xr[i][0] = a.x; xr[i][1] = a.y; xr[i][2] = a.z; xr[i][3] = a.w;
-            xr[i][4] = b.x; xr[i][5] = b.y; xr[i][6] = b.z; xr[i][7] = b.w;
+        if (c * CE < p.kw) {
+            const float4 *xp = reinterpret_cast<const float4 *>(p.x + (size_t)ks * p.kw + (size_t)c * CE);
+#pragma unroll
+            for (int q = 0; q < CE / 4; ++q) {
+                const float4 a = xp[q];
+                xr[i][4 * q] = a.x; xr[i][4 * q + 1] = a.y; xr[i][4 * q + 2] = a.z; xr[i][4 * q + 3] = a.w;
+            }
         } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) xr[i][e] = 0.f;
+            for (int e = 0; e < CE; ++e) xr[i][e] = 0.f;
         }
         if (NORM) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
-            const uint4 g = gr[i];
-            xr[i][0] *= bf16_lo(g.x); xr[i][1] *= bf16_hi(g.x);
-            xr[i][2] *= bf16_lo(g.y); xr[i][3] *= bf16_hi(g.y);
-            xr[i][4] *= bf16_lo(g.z); xr[i][5] *= bf16_hi(g.z);
-            xr[i][6] *= bf16_lo(g.w); xr[i][7] *= bf16_hi(g.w);
+            for (int e = 0; e < CE; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
+#pragma unroll
+            for (int h = 0; h < CE / 8; ++h) {
+                const uint4 g = gr[i][h];
+                xr[i][8 * h + 0] *= bf16_lo(g.x); xr[i][8 * h + 1] *= bf16_hi(g.x);
+                xr[i][8 * h + 2] *= bf16_lo(g.y); xr[i][8 * h + 3] *= bf16_hi(g.y);
+                xr[i][8 * h + 4] *= bf16_lo(g.z); xr[i][8 * h + 5] *= bf16_hi(g.z);
+                xr[i][8 * h + 6] *= bf16_lo(g.w); xr[i][8 * h + 7] *= bf16_hi(g.w);
+            }
         }
     }
     if (NORM) {
@@ -237,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     uint32_t phase = 0;
     bool ok = true, done = false;
     float inv = 1.f;
-    const uint32_t slice_off = (uint32_t)ks * (uint32_t)p.kw * 2u;
+    const uint32_t slice_off = (uint32_t)ks * (uint32_t)p.kw * (uint32_t)WB;
     const int t = threadIdx.x;
     const int fold_unit = (MODE == kGemvSwiglu) ? (p.rps >> 1) : p.rps;   // outputs per stage
     const int tj = t / fold_unit, tr = t % fold_unit;                      // this thread's (stage in block, output in stage)
@@ -271,12 +317,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
                     const int c = lane + 32 * i;
                     w0[i] = make_uint4(0, 0, 0, 0);
                     w1[i] = make_uint4(0, 0, 0, 0);
-                    if (c * 8 < p.kw) {
+                    if (c * CE < p.kw) {
                         w0[i] = lds128(rbase0 + (uint32_t)c * 16u);
                         w1[i] = lds128(rbase1 + (uint32_t)c * 16u);
                     }
                 }
-                float s0 = dot_slice<J>(w0, xr), s1 = dot_slice<J>(w1, xr);
+                float s0, s1;
+                if constexpr (WB == 2) { s0 = dot_slice<J>(w0, xr); s1 = dot_slice<J>(w1, xr); }
+                else { s0 = dot_slice_fp8<J>(w0, xr); s1 = dot_slice_fp8<J>(w1, xr); }
                 // joint reduction: lanes 0-15 end up with row 0, lanes 16-31 with row 1
                 const bool upper = (lane & 16) != 0;
                 float keep = upper ? s1 : s0;
@@ -308,6 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
                     float g = 0.f, u = 0.f;
                     for (int k = 0; k < ksplit; ++k) { g += part[buf][r][k]; u += part[buf][r + 1][k]; }
                     g *= inv; u *= inv;
+                    if (WB == 1) { g *= p.wscale[row0 + 2 * tr]; u *= p.wscale[row0 + 2 * tr + 1]; }
                     p.y[(row0 >> 1) + tr] = g / (1.f + __expf(-g)) * u;
                 }
             } else if (row0 + tr < p.n_out) {
@@ -315,6 +364,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
                 for (int k = 0; k < ksplit; ++k) v += part[buf][tj * p.rps + tr][k];
                 v *= inv;
                 const int row = row0 + tr;
+                if (WB == 1) v *= p.wscale[row];
                 // residual: each element is touched by exactly one thread of one CTA per launch, so a reduction
                 // without return value gives the same sum as load-add-store and exposes no load latency
                 if (MODE == kGemvResidual) atomicAdd(p.y + row, v);
@@ -375,9 +425,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
     }
 }
 
-template <int J, int MODE, bool NORM>
+template <int J, int MODE, bool NORM, int WB>
 cudaError_t launch_j(const LaunchCtx &lc, const StreamParams &p, int grid, size_t smem) {
-    auto kern = gemv_stream_kernel<J, MODE, NORM>;
+    auto kern = gemv_stream_kernel<J, MODE, NORM, WB>;
     static unsigned long long attr_done = 0;   // per instantiation, one bit per device
     if (cudaError_t e = ensure_dynamic_smem(kern, kRingBytes, &attr_done); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -395,14 +445,23 @@ cudaError_t launch_j(const LaunchCtx &lc, const StreamParams &p, int grid, size_
 }
 
 template <int MODE, bool NORM>
-cudaError_t launch_mode(const LaunchCtx &lc, const StreamParams &p, int J, int grid, size_t smem) {
+cudaError_t launch_mode(const LaunchCtx &lc, const StreamParams &p, int J, int grid, size_t smem, int wb) {
+    if (wb == 1) {   // FP8: a chunk carries 16 weights, so half as many chunks cover a slice
+        switch (J) {
+            case 1: return launch_j<1, MODE, NORM, 1>(lc, p, grid, smem);
+            case 2: return launch_j<2, MODE, NORM, 1>(lc, p, grid, smem);
+            case 3: return launch_j<3, MODE, NORM, 1>(lc, p, grid, smem);
+            case 4: return launch_j<4, MODE, NORM, 1>(lc, p, grid, smem);
+        }
+        return cudaErrorInvalidValue;
+    }
     switch (J) {
-        case 1: return launch_j<1, MODE, NORM>(lc, p, grid, smem);
-        case 2: return launch_j<2, MODE, NORM>(lc, p, grid, smem);
-        case 3: return launch_j<3, MODE, NORM>(lc, p, grid, smem);
-        case 4: return launch_j<4, MODE, NORM>(lc, p, grid, smem);
-        case 5: case 6: return launch_j<6, MODE, NORM>(lc, p, grid, smem);
-        case 7: case 8: return launch_j<8, MODE, NORM>(lc, p, grid, smem);
+        case 1: return launch_j<1, MODE, NORM, 2>(lc, p, grid, smem);
+        case 2: return launch_j<2, MODE, NORM, 2>(lc, p, grid, smem);
+        case 3: return launch_j<3, MODE, NORM, 2>(lc, p, grid, smem);
+        case 4: return launch_j<4, MODE, NORM, 2>(lc, p, grid, smem);
+        case 5: case 6: return launch_j<6, MODE, NORM, 2>(lc, p, grid, smem);
+        case 7: case 8: return launch_j<8, MODE, NORM, 2>(lc, p, grid, smem);
     }
     return cudaErrorInvalidValue;
 }
@@ -411,19 +470,21 @@ cudaError_t launch_mode(const LaunchCtx &lc, const StreamParams &p, int J, int g
 // (each is one bulk copy; the per-stage handshake amortises and the copy engine's request rate never binds),
 // an even number of rows per warp per stage (rows are processed in pairs), K slices of 2 KB or more, an even row
 // count per stage when rows pair up as gate/up, and then the best balance over the SMs.
-bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int *ksplit_out, int *rps_out) {
+bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int wb, int *ksplit_out, int *rps_out) {
     double best = -1.0;
 #ifdef NNC_TUNING
     if (const char *g = getenv("NNC_GEMV_GEOM")) {   // "ksplit,rps": tuning builds only
         if (sscanf(g, "%d,%d", ksplit_out, rps_out) == 2) return true;
     }
 #endif
-    const int row_bytes = K * 2;
+    const int row_bytes = K * wb;
+    const int ce = 16 / wb;                      // weights per 16-byte chunk
+    const int max_chunks = wb == 2 ? 8 : 4;      // chunks per lane the kernel is instantiated for
     for (int ks = 8; ks >= 1; ks >>= 1) {
-        if (K % (8 * ks)) continue;
+        if (K % (ce * ks)) continue;
         const int kw = K / ks;
-        if ((kw + 255) / 256 > 8) continue;     // at most 8 chunks per lane
-        if (kw * 2 < 512 && ks > 1) continue;
+        if ((kw + 32 * ce - 1) / (32 * ce) > max_chunks) continue;
+        if (kw * wb < 512 && ks > 1) continue;
         const int gpi = kConsumerWarps / ks;
         for (int rps = gpi; rps <= kBlockRows; rps += gpi) {
             if (pairs && (rps & 1)) continue;
@@ -439,8 +500,8 @@ bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int *ksplit_out, 
             if (bytes < 8192) score *= 0.80;
             else if (bytes < 16384) score *= 0.90;
             else if (bytes < 24576) score *= 0.95;
-            if (kw * 2 < 1024) score *= 0.90;
-            else if (kw * 2 < 2048) score *= 0.93;
+            if (kw * wb < 1024) score *= 0.90;
+            else if (kw * wb < 2048) score *= 0.93;
             if (score > best) { best = score; *ksplit_out = ks; *rps_out = rps; }
         }
     }
@@ -449,34 +510,24 @@ bool pick_geometry(int n_out, int K, int sm_count, bool pairs, int *ksplit_out, 
 
 }  // namespace
 
-bool gemv_stream_geometry(int n_out, int n_in, int sm_count, int mode, GemvGeom *out) {
-    if (!gemv_stream_supported(n_out, n_in, mode)) return false;
-    GemvGeom g;
-    g.n_out = n_out; g.K = n_in;
-    if (!pick_geometry(n_out, n_in, sm_count, mode == kGemvSwiglu, &g.ksplit, &g.rps)) return false;
-    g.kw = n_in / g.ksplit;
-    g.n_stages = (n_out + g.rps - 1) / g.rps;
-    const int j = (g.kw + 255) / 256;
-    g.J = j <= 4 ? j : (j <= 6 ? 6 : 8);
-    *out = g;
-    return true;
-}
-
-bool gemv_stream_supported(int n_out, int n_in, int mode) {
+bool gemv_stream_supported(int n_out, int n_in, int mode, int wb) {
     int ks, rps;
-    if (n_out < 1 || n_in % 8 || n_in < 64 || (mode == kGemvSwiglu && n_out % 2)) return false;
-    return pick_geometry(n_out, n_in, 148, mode == kGemvSwiglu, &ks, &rps);
+    if (n_out < 1 || n_in % (16 / wb) || n_in < 64 || (mode == kGemvSwiglu && n_out % 2)) return false;
+    return pick_geometry(n_out, n_in, 148, mode == kGemvSwiglu, wb, &ks, &rps);
 }
 
-cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr) {
-    if (!gemv_stream_supported(n_out, n_in, mode)) return cudaErrorInvalidValue;
+cudaError_t launch_gemv_stream(const LaunchCtx &lc, const void *W, const float *wscale, int wb, const float *x, float *y,
+                               int n_out, int n_in, const bf16 *gain, float eps, int mode, const ArgmaxScratch *am,
+                               uint32_t *ctr) {
+    if ((wb != 1 && wb != 2) || (wb == 1 && !wscale)) return cudaErrorInvalidValue;
+    if (!gemv_stream_supported(n_out, n_in, mode, wb)) return cudaErrorInvalidValue;
     StreamParams p;
-    if (!pick_geometry(n_out, n_in, lc.sm_count, mode == kGemvSwiglu, &p.ksplit, &p.rps)) return cudaErrorInvalidValue;
+    if (!pick_geometry(n_out, n_in, lc.sm_count, mode == kGemvSwiglu, wb, &p.ksplit, &p.rps)) return cudaErrorInvalidValue;
     p.W = reinterpret_cast<const uint8_t *>(W);
+    p.wscale = wscale;
     p.x = x; p.y = y; p.gain = gain; p.eps = eps; p.n_out = n_out; p.K = n_in;
     p.kw = n_in / p.ksplit;
-    const int stage_bytes = p.rps * n_in * 2;
+    const int stage_bytes = p.rps * n_in * wb;
     int S = kRingBytes / stage_bytes;
     if (S > kMaxStages) S = kMaxStages;
     if (S < 2) return cudaErrorInvalidValue;
@@ -497,17 +548,18 @@ cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *
     p.ctr = n_runs > lc.sm_count ? ctr : nullptr;
     if (mode == kGemvLogits && grid > kArgmaxMaxBlocks) grid = kArgmaxMaxBlocks;
     const size_t smem = (size_t)S * stage_bytes;
-    const int J = (p.kw + 255) / 256;
+    const int ce32 = 32 * (16 / wb);
+    const int J = (p.kw + ce32 - 1) / ce32;
     const bool norm = gain != nullptr;
     switch (mode) {
         case kGemvStore:
-            return norm ? launch_mode<kGemvStore, true>(lc, p, J, grid, smem) : launch_mode<kGemvStore, false>(lc, p, J, grid, smem);
+            return norm ? launch_mode<kGemvStore, true>(lc, p, J, grid, smem, wb) : launch_mode<kGemvStore, false>(lc, p, J, grid, smem, wb);
         case kGemvResidual:
-            return norm ? launch_mode<kGemvResidual, true>(lc, p, J, grid, smem) : launch_mode<kGemvResidual, false>(lc, p, J, grid, smem);
+            return norm ? launch_mode<kGemvResidual, true>(lc, p, J, grid, smem, wb) : launch_mode<kGemvResidual, false>(lc, p, J, grid, smem, wb);
         case kGemvSwiglu:
-            return norm ? launch_mode<kGemvSwiglu, true>(lc, p, J, grid, smem) : launch_mode<kGemvSwiglu, false>(lc, p, J, grid, smem);
+            return norm ? launch_mode<kGemvSwiglu, true>(lc, p, J, grid, smem, wb) : launch_mode<kGemvSwiglu, false>(lc, p, J, grid, smem, wb);
         case kGemvLogits:
-            return norm ? launch_mode<kGemvLogits, true>(lc, p, J, grid, smem) : launch_mode<kGemvLogits, false>(lc, p, J, grid, smem);
+            return norm ? launch_mode<kGemvLogits, true>(lc, p, J, grid, smem, wb) : launch_mode<kGemvLogits, false>(lc, p, J, grid, smem, wb);
     }
     return cudaErrorInvalidValue;
 }

@@ -25,12 +25,21 @@ constexpr int kHostLogitRows = 64;  // rows of logits the *_host variants can st
 
 struct LayerW {
     bf16 *wqkv, *wo, *wgu, *wd, *g_in, *g_post, *g_q, *g_k;
+    // fp16 copies for the prompt-phase GEMMs (null without them), each scaled by a power of two; sc_* point at the
+    // DEVICE pair {2^e, 2^-e} of the matrix
+    void *wo16, *wgu16, *wd16;
+    float *sc_o, *sc_gu, *sc_d;
+    // weight_format 1: FP8 E4M3 codes and per-row scales of the four matrices (null otherwise)
+    uint8_t *q_qkv, *q_o, *q_gu, *q_d;
+    float *s_qkv, *s_o, *s_gu, *s_d;
 };
 
 struct Plan {
     size_t total = 0;
     // offsets
-    std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk;
+    std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk, l_wo16, l_wgu16, l_wd16;
+    std::vector<size_t> l_q8, l_s8;   // FP8: codes of the four matrices back to back, then their row scales
+    size_t f16_scales, f16_word, lm_q8, lm_s8;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
     size_t gemv_ctr, gemm_part, gemm_tickets, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
     size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
@@ -52,8 +61,14 @@ bool valid_config(const nnc_config &c) {
     if (c.hidden % 64 || c.intermediate % 64 || c.vocab % 8) return false;
     if ((size_t)c.intermediate * 4 > 200 * 1024 || (size_t)c.n_q_heads * 128 * 4 > 200 * 1024) return false;
     if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return false;
+    if (c.tc_operands < 0 || c.tc_operands > 2) return false;
+    if (c.weight_format < 0 || c.weight_format > 1) return false;
+    if (c.weight_format == 1 && (c.hidden % 128 || c.intermediate % 128)) return false;   // the FP8 GEMV's K slices
     return true;
 }
+
+// fp16 copies of Wo, Wgate/up and Wdown exist when the model may see calls of more than 128 tokens in operand mode 0
+bool wants_f16_copies(const nnc_config &c) { return c.tc_operands == 0 && c.max_tokens > 128; }
 
 void make_plan(const nnc_config &c, Plan &p) {
     const size_t H = c.hidden, qd = (size_t)c.n_q_heads * 128, kd = (size_t)c.n_kv_heads * 128, I = c.intermediate;
@@ -67,7 +82,20 @@ void make_plan(const nnc_config &c, Plan &p) {
         p.l_gpost.push_back(p.take(H * 2));
         p.l_gq.push_back(p.take(128 * 2));
         p.l_gk.push_back(p.take(128 * 2));
+        if (c.weight_format == 1) {
+            p.l_q8.push_back(p.take(qkvd * H + H * qd + 2 * I * H + H * I));
+            p.l_s8.push_back(p.take((qkvd + H + 2 * I + H) * sizeof(float)));
+        }
+        if (wants_f16_copies(c)) {
+            p.l_wo16.push_back(p.take(H * qd * 2));
+            p.l_wgu16.push_back(p.take(2 * I * H * 2));
+            p.l_wd16.push_back(p.take(H * I * 2));
+        }
     }
+    p.lm_q8 = p.take(c.weight_format == 1 ? V * H : 0);
+    p.lm_s8 = p.take(c.weight_format == 1 ? V * sizeof(float) : 0);
+    p.f16_scales = p.take((size_t)c.n_layers * 3 * 2 * sizeof(float));
+    p.f16_word = p.take(4);
     p.embed = p.take(V * H * 2);
     p.lm_head = c.tie_embeddings ? p.embed : p.take(V * H * 2);
     p.g_final = p.take(H * 2);
@@ -121,7 +149,10 @@ struct nnc_model {
     int32_t *d_len, *d_status, *d_tokens, *d_argmax;
     float *xt, *qkvt, *logits_stage;
     bf16 *hb, *ob, *ab;
-    bf16 *hb_lo, *ob_lo, *ab_lo;  // bf16 rounding residuals of the GEMM activations (null in fast mode)
+    bf16 *hb_lo, *ob_lo, *ab_lo;  // bf16 rounding residuals of the GEMM activations (null in the one-term mode)
+    bool f16_copies;              // the layers hold fp16 copies of Wo, Wgate/up, Wdown
+    uint8_t *lm_q8;               // weight_format 1: FP8 codes and row scales of the lm_head (null otherwise)
+    float *lm_s8;
     int len;
     float *taps;
     bool pdl;
@@ -168,13 +199,14 @@ int layer_decode_b1(nnc_model *m, int l, const LaunchCtx &lc, int n_splits) {
     bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
     bf16 *vc = m->vcache + (size_t)l * m->kv_layer_stride();
     uint32_t *ctr = m->gemv_ctr + (size_t)l * 16;
-    NNC_CUDA(m, launch_gemv(lc, w.wqkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr, ctr));
+    const bool q8 = c.weight_format == 1;
+    NNC_CUDA(m, launch_gemv(lc, q8 ? (const void *)w.q_qkv : w.wqkv, w.s_qkv, m->x, m->qkv, m->qkvd(), c.hidden, w.g_in, c.rms_eps, kGemvStore, nullptr, ctr));
     const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
     NNC_CUDA(m, launch_attn_decode(lc, m->qkv, m->qkvd(), kc, vc, m->attn_out, nullptr, nullptr, m->qd(), m->part, m->tickets,
                                    m->d_len, 1, 1, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
-    NNC_CUDA(m, launch_gemv(lc, w.wo, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr, ctr + 4));
-    NNC_CUDA(m, launch_gemv(lc, w.wgu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr, ctr + 8));
-    NNC_CUDA(m, launch_gemv(lc, w.wd, m->act, m->x, c.hidden, c.intermediate, nullptr, 0.f, kGemvResidual, nullptr, ctr + 12));
+    NNC_CUDA(m, launch_gemv(lc, q8 ? (const void *)w.q_o : w.wo, w.s_o, m->attn_out, m->x, c.hidden, m->qd(), nullptr, 0.f, kGemvResidual, nullptr, ctr + 4));
+    NNC_CUDA(m, launch_gemv(lc, q8 ? (const void *)w.q_gu : w.wgu, w.s_gu, m->x, m->act, 2 * c.intermediate, c.hidden, w.g_post, c.rms_eps, kGemvSwiglu, nullptr, ctr + 8));
+    NNC_CUDA(m, launch_gemv(lc, q8 ? (const void *)w.q_d : w.wd, w.s_d, m->act, m->x, c.hidden, c.intermediate, nullptr, 0.f, kGemvResidual, nullptr, ctr + 12));
     return NNC_OK;
 }
 
@@ -189,7 +221,7 @@ int decode_b1_launches(nnc_model *m, const int32_t *tokens, float *logits, int32
     }
     ArgmaxScratch am = m->am;
     am.out = argmax;
-    NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->x, logits, c.vocab, c.hidden, m->g_final, c.rms_eps, kGemvLogits, &am,
+    NNC_CUDA(m, launch_gemv(lc, m->lm_q8 ? (const void *)m->lm_q8 : m->lm_head, m->lm_s8, m->x, logits, c.vocab, c.hidden, m->g_final, c.rms_eps, kGemvLogits, &am,
                             m->gemv_ctr + (size_t)c.n_layers * 16));
     NNC_CUDA(m, launch_add_len(lc, m->d_len, 1));
     return NNC_OK;
@@ -202,6 +234,9 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
     LaunchCtx lc = ctx(m, m->pdl);
     NNC_CUDA(m, launch_embed(lc, m->embed, tokens, m->xt, R, H, c.vocab, m->taps));
     const int n_splits = attn_decode_splits(m->sm_count, batch, c.n_kv_heads, c.max_seq);
+    // prompt-phase calls of more than 128 tokens: attention output, MLP input and SwiGLU output travel as one fp16 term
+    // and meet the fp16 weight copies; the QKV input keeps two bf16 terms (see nnc_config::tc_operands)
+    const bool f16 = m->f16_copies && T > 1 && R > 128;
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW &w = m->layers[l];
         bf16 *kc = m->kcache + (size_t)l * m->kv_layer_stride();
@@ -215,12 +250,19 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
         } else {
             NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
                                                    c.n_kv_heads, c.max_seq, m->d_len, nullptr));
-            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, m->ob_lo, false, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len));
+            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, f16 ? nullptr : m->ob_lo, f16, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len));
         }
-        NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
-        NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
-        NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wgu, m->ab, m->ab_lo, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status, &m->gemm_scratch));
-        NNC_CUDA(m, launch_gemm(lc, m->ab, m->ab_lo, w.wd, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
+        if (f16) {
+            NNC_CUDA(m, launch_gemm(lc, m->ob, nullptr, (const bf16 *)w.wo16, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, nullptr, true, w.sc_o + 1));
+            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, nullptr, R, H, c.rms_eps, 0, 1, true));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, nullptr, (const bf16 *)w.wgu16, m->ab, nullptr, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status, nullptr, true, w.sc_gu + 1));
+            NNC_CUDA(m, launch_gemm(lc, m->ab, nullptr, (const bf16 *)w.wd16, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status, nullptr, true, w.sc_d + 1));
+        } else {
+            NNC_CUDA(m, launch_gemm(lc, m->ob, m->ob_lo, w.wo, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
+            NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, w.g_post, m->hb, m->hb_lo, R, H, c.rms_eps, 0, 1));
+            NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, w.wgu, m->ab, m->ab_lo, R, 2 * I, H, I, kEpiSwigluBf16, m->d_status, &m->gemm_scratch));
+            NNC_CUDA(m, launch_gemm(lc, m->ab, m->ab_lo, w.wd, m->xt, nullptr, R, H, I, H, kEpiAccumF32, m->d_status, &m->gemm_scratch));
+        }
         if (m->taps) NNC_CUDA(m, launch_copy_f32(lc, m->xt, m->taps + (size_t)(l + 1) * R * H, (size_t)R * H));
     }
     if (logits) {
@@ -229,7 +271,7 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
             NNC_CUDA(m, launch_gemm(lc, m->hb, m->hb_lo, m->lm_head, logits, nullptr, R, c.vocab, H, c.vocab, kEpiStoreF32, m->d_status, &m->gemm_scratch));
         } else if (batch == 1) {
             // last position only: the streaming GEMV keeps the activation in fp32
-            NNC_CUDA(m, launch_gemv(lc, m->lm_head, m->xt + (size_t)(T - 1) * H, logits, c.vocab, H, m->g_final, c.rms_eps,
+            NNC_CUDA(m, launch_gemv(lc, m->lm_q8 ? (const void *)m->lm_q8 : m->lm_head, m->lm_s8, m->xt + (size_t)(T - 1) * H, logits, c.vocab, H, m->g_final, c.rms_eps,
                                     kGemvLogits, nullptr));
         } else {
             NNC_CUDA(m, launch_rmsnorm_rows(lc, m->xt, m->g_final, m->hb, m->hb_lo, batch, H, c.rms_eps, T - 1, T));
@@ -300,7 +342,20 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
             w.wqkv = (bf16 *)at(p.l_wqkv[l]); w.wo = (bf16 *)at(p.l_wo[l]); w.wgu = (bf16 *)at(p.l_wgu[l]);
             w.wd = (bf16 *)at(p.l_wd[l]); w.g_in = (bf16 *)at(p.l_gin[l]); w.g_post = (bf16 *)at(p.l_gpost[l]);
             w.g_q = (bf16 *)at(p.l_gq[l]); w.g_k = (bf16 *)at(p.l_gk[l]);
+            w.wo16 = w.wgu16 = w.wd16 = nullptr;
+            w.sc_o = (float *)at(p.f16_scales) + (size_t)l * 6;
+            w.sc_gu = w.sc_o + 2; w.sc_d = w.sc_o + 4;
+            if (wants_f16_copies(c)) { w.wo16 = at(p.l_wo16[l]); w.wgu16 = at(p.l_wgu16[l]); w.wd16 = at(p.l_wd16[l]); }
+            w.q_qkv = w.q_o = w.q_gu = w.q_d = nullptr;
+            w.s_qkv = w.s_o = w.s_gu = w.s_d = nullptr;
+            if (c.weight_format == 1) {
+                const size_t qkvd = (size_t)m->qkvd(), Hs = c.hidden, qds = m->qd(), Is = c.intermediate;
+                w.q_qkv = (uint8_t *)at(p.l_q8[l]); w.q_o = w.q_qkv + qkvd * Hs; w.q_gu = w.q_o + Hs * qds; w.q_d = w.q_gu + 2 * Is * Hs;
+                w.s_qkv = (float *)at(p.l_s8[l]); w.s_o = w.s_qkv + qkvd; w.s_gu = w.s_o + Hs; w.s_d = w.s_gu + 2 * Is;
+            }
         }
+        m->lm_q8 = c.weight_format == 1 ? (uint8_t *)at(p.lm_q8) : nullptr;
+        m->lm_s8 = c.weight_format == 1 ? (float *)at(p.lm_s8) : nullptr;
         m->embed = (bf16 *)at(p.embed); m->lm_head = (bf16 *)at(p.lm_head); m->g_final = (bf16 *)at(p.g_final);
         m->kcache = (bf16 *)at(p.kcache); m->vcache = (bf16 *)at(p.vcache); m->rope = (float *)at(p.rope);
         m->x = (float *)at(p.x); m->qkv = (float *)at(p.qkv); m->attn_out = (float *)at(p.attn_out);
@@ -312,7 +367,8 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
         m->d_tokens = (int32_t *)at(p.d_tokens); m->d_argmax = (int32_t *)at(p.d_argmax);
         m->xt = (float *)at(p.xt); m->hb = (bf16 *)at(p.hb); m->qkvt = (float *)at(p.qkvt);
         m->ob = (bf16 *)at(p.ob); m->ab = (bf16 *)at(p.ab); m->logits_stage = (float *)at(p.logits_stage);
-        const bool fast = c.fast_bf16_activations != 0;
+        const bool fast = c.tc_operands == 2;
+        m->f16_copies = wants_f16_copies(c);
         m->hb_lo = fast ? nullptr : (bf16 *)at(p.hb_lo);
         m->ob_lo = fast ? nullptr : (bf16 *)at(p.ob_lo);
         m->ab_lo = fast ? nullptr : (bf16 *)at(p.ab_lo);
@@ -338,11 +394,25 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
             NNC_CUDA(m, cudaMemcpyAsync(w.g_post, s.g_post, (size_t)H * 2, cudaMemcpyDeviceToDevice, m->stream));
             NNC_CUDA(m, cudaMemcpyAsync(w.g_q, s.g_q, 256, cudaMemcpyDeviceToDevice, m->stream));
             NNC_CUDA(m, cudaMemcpyAsync(w.g_k, s.g_k, 256, cudaMemcpyDeviceToDevice, m->stream));
+            if (c.weight_format == 1) {   // quantise; the bf16 store keeps the dequantised values
+                NNC_CUDA(m, launch_quantise_rows_e4m3(lc, w.wqkv, w.q_qkv, w.s_qkv, w.wqkv, m->qkvd(), H));
+                NNC_CUDA(m, launch_quantise_rows_e4m3(lc, w.wo, w.q_o, w.s_o, w.wo, H, qd));
+                NNC_CUDA(m, launch_quantise_rows_e4m3(lc, w.wgu, w.q_gu, w.s_gu, w.wgu, 2 * I, H));
+                NNC_CUDA(m, launch_quantise_rows_e4m3(lc, w.wd, w.q_d, w.s_d, w.wd, H, I));
+            }
+            if (m->f16_copies) {
+                uint32_t *word = (uint32_t *)at(p.f16_word);
+                NNC_CUDA(m, launch_to_f16_scaled(lc, w.wo, w.wo16, (size_t)H * qd, w.sc_o, word));
+                NNC_CUDA(m, launch_to_f16_scaled(lc, w.wgu, w.wgu16, (size_t)2 * I * H, w.sc_gu, word));
+                NNC_CUDA(m, launch_to_f16_scaled(lc, w.wd, w.wd16, (size_t)H * I, w.sc_d, word));
+            }
         }
         NNC_CUDA(m, launch_copy_rows(lc, (const bf16 *)weights->embed, m->embed, c.vocab, H, 0, 1, 0, 1));
         if (!c.tie_embeddings)
             NNC_CUDA(m, launch_copy_rows(lc, (const bf16 *)weights->lm_head, m->lm_head, c.vocab, H, 0, 1, 0, 1));
         NNC_CUDA(m, cudaMemcpyAsync(m->g_final, weights->g_final, (size_t)H * 2, cudaMemcpyDeviceToDevice, m->stream));
+        if (c.weight_format == 1)   // a tied embedding is this same matrix: the gather then reads the dequantised rows
+            NNC_CUDA(m, launch_quantise_rows_e4m3(lc, m->lm_head, m->lm_q8, m->lm_s8, m->lm_head, c.vocab, H));
 
         // ---- RoPE table: cos/sin of p * theta^(-2i/128) in double, rounded once to fp32 ----
         {
@@ -673,6 +743,38 @@ int nnc_op_gemm_splitk(const void *X, const void *X_lo, const void *W, void *Y, 
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 
+int nnc_op_gemm_f16(const void *X, const void *W, float *Y, int32_t T, int32_t n_out, int32_t n_in, int32_t accumulate,
+                    const float *out_scale, void *cuda_stream) {
+    if (!X || !W || !Y) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_gemm(lc, (const bf16 *)X, nullptr, (const bf16 *)W, Y, nullptr, T, n_out, n_in, n_out,
+                                accumulate ? kEpiAccumF32 : kEpiStoreF32, lc.status, nullptr, true, out_scale);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
+int nnc_op_gemm_swiglu_f16(const void *X, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,
+                           const float *out_scale, void *cuda_stream) {
+    if (!X || !W || !Y || n_out % 2) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_gemm(lc, (const bf16 *)X, nullptr, (const bf16 *)W, Y, nullptr, T, n_out, n_in, n_out / 2,
+                                kEpiSwigluBf16, lc.status, nullptr, true, out_scale);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
+int nnc_op_to_f16_scaled(const void *src, void *dst, size_t n, float *scales, uint32_t *scratch_word, void *cuda_stream) {
+    if (!src || !dst || !scales || !scratch_word || n == 0 || n % 8) return NNC_ERR_INVALID_ARG;
+    if (((uintptr_t)src | (uintptr_t)dst) & 15) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_to_f16_scaled(lc, (const bf16 *)src, dst, n, scales, scratch_word);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
 int nnc_op_status(int32_t *status_out) {
     if (!status_out) return NNC_ERR_INVALID_ARG;
     int zero = 0;
@@ -693,8 +795,31 @@ int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t 
     if (cudaGetSymbolAddress((void **)&ctrs, g_op_gemv_ctr) != cudaSuccess) return NNC_ERR_CUDA;
     static unsigned rotation = 0;   // call sites taken in turn; atomic so that concurrent host threads get distinct ones
     const unsigned site = __atomic_fetch_add(&rotation, 1u, __ATOMIC_RELAXED) % 8;
-    cudaError_t e = launch_gemv(lc, (const bf16 *)W, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr,
-                                ctrs + 4 * site);
+    cudaError_t e = launch_gemv(lc, W, nullptr, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr, ctrs + 4 * site);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
+int nnc_op_gemv_fp8(const void *codes, const float *scales, const float *x, float *y, int32_t n_out, int32_t n_in,
+                    const void *gain, float eps, int32_t mode, void *cuda_stream) {
+    const bool chained = (mode & NNC_GEMV_CHAINED) != 0;
+    mode &= ~NNC_GEMV_CHAINED;
+    if (!codes || !scales || !x || !y || mode < 0 || mode > 2) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    lc.pdl = chained;
+    cudaError_t e = launch_gemv(lc, codes, scales, x, y, n_out, n_in, (const bf16 *)gain, eps, mode, nullptr, nullptr);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
+int nnc_op_quantise_rows_e4m3(const void *W, void *codes, float *scales, void *dequant, int32_t n_out, int32_t n_in,
+                              void *cuda_stream) {
+    if (!W || !codes || !scales) return NNC_ERR_INVALID_ARG;
+    if (((uintptr_t)W | (uintptr_t)codes | (uintptr_t)dequant) & 15) return NNC_ERR_INVALID_ARG;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_quantise_rows_e4m3(lc, (const bf16 *)W, (uint8_t *)codes, scales, (bf16 *)dequant, n_out, n_in);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }

@@ -60,22 +60,23 @@ struct ArgmaxScratch {
 
 // ctr (nullable): two zeroed words owned by this call site, used by the streaming form to hand out work
 // dynamically; a call site may be launched again only after ~4 later GEMVs of the same stream have started.
-cudaError_t launch_gemv(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
+// Weights: bf16 W[n_out][n_in] (wscale null), or FP8 E4M3 codes W[n_out][n_in] with wscale[n_out] (one scale per row).
+cudaError_t launch_gemv(const LaunchCtx &lc, const void *W, const float *wscale, const float *x, float *y, int n_out, int n_in,
                         const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr = nullptr);
 
-// streaming form (decode_gemv_stream.cu): n_in a multiple of 8 up to 16384 (8192 for SwiGLU); launch_gemv uses it
-// whenever the shape allows and falls back to the plain-load kernel otherwise
-bool gemv_stream_supported(int n_out, int n_in, int mode);
-cudaError_t launch_gemv_stream(const LaunchCtx &lc, const bf16 *W, const float *x, float *y, int n_out, int n_in,
-                               const bf16 *gain, float eps, int mode, const ArgmaxScratch *am, uint32_t *ctr);
+// streaming form (decode_gemv_stream.cu): n_in a multiple of 8 up to 16384 (8192 for SwiGLU) for bf16, a multiple of
+// 16 for FP8 (wb = bytes per weight); launch_gemv uses it whenever the shape allows and, for bf16, falls back to the
+// plain-load kernel otherwise
+bool gemv_stream_supported(int n_out, int n_in, int mode, int wb = 2);
+cudaError_t launch_gemv_stream(const LaunchCtx &lc, const void *W, const float *wscale, int wb, const float *x, float *y,
+                               int n_out, int n_in, const bf16 *gain, float eps, int mode, const ArgmaxScratch *am,
+                               uint32_t *ctr);
 
-// Slicing of one matrix for the streaming GEMV: consumer warps per row, columns per warp slice, rows per stage,
-// stages in the matrix, 16-byte chunks per lane per slice (rounded up to an instantiated value).
-struct GemvGeom {
-    int n_out, K;
-    int ksplit, kw, rps, n_stages, J;
-};
-bool gemv_stream_geometry(int n_out, int n_in, int sm_count, int mode, GemvGeom *out);
+// FP8 E4M3 row quantisation (repack.cu): codes[n_out][n_in], scales[n_out] = 2^e with e the smallest integer such that
+// the row's largest magnitude is at most 448 * 2^e; round to nearest even, saturating.  If dequant is not null it
+// receives code * 2^e as bf16 (exact); it may alias W.
+cudaError_t launch_quantise_rows_e4m3(const LaunchCtx &lc, const bf16 *W, uint8_t *codes, float *scales, bf16 *dequant,
+                                      int n_out, int n_in);
 
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,

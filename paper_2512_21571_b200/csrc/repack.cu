@@ -4,7 +4,7 @@
 //
 // Also here: the fp16 copy of a bf16 matrix that the prompt-phase GEMMs multiply with fp16 activations.  fp16 has more
 // mantissa bits than bf16 but a narrow exponent range, so the copy holds W * 2^e with e chosen per matrix such that
-// the largest magnitude lands in [2^14, 2^15): every weight down to 2^-38 of the largest one converts exactly (the 8
+// the largest magnitude lands in [2^14, 2^15): every weight down to 2^-32 of the largest one converts exactly (the 8
 // significant bits of a bf16 value fit, and the scaling is a power of two); smaller ones round on the fp16 subnormal
 // grid, an error below 2^-39 of the largest weight.  The GEMM epilogue multiplies by 2^-e.
 #include <cuda_fp16.h>
@@ -73,7 +73,82 @@ __global__ void to_f16_scaled_kernel(const uint4 *__restrict__ src, uint4 *__res
     }
 }
 
+// FP8 E4M3 row quantisation, one block per row: e = the smallest integer with max|w| <= 448 * 2^e; codes = round to
+// nearest even of w * 2^-e onto the E4M3 grid (saturating; the hardware conversion); scale = 2^e.  The scaling by a
+// power of two is exact, so host and device reach the same codes bit for bit.
+__global__ void __launch_bounds__(256)
+quantise_rows_e4m3_kernel(const bf16 *W, uint8_t *__restrict__ codes, float *__restrict__ scales,
+                          bf16 *dequant /* may alias W: every thread reads a chunk before it writes that chunk */, int n_in) {
+    __shared__ uint32_t red[8];
+    const size_t row = blockIdx.x;
+    const uint4 *src = reinterpret_cast<const uint4 *>(W + row * n_in);
+    const int n8 = n_in / 8;
+    uint32_t m = 0;
+    for (int i = threadIdx.x; i < n8; i += 256) {
+        const uint4 v = src[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t a = (w[k] << 16) & 0x7fffffffu, b = w[k] & 0x7fff0000u;
+            if (a <= 0x7f800000u && a > m) m = a;
+            if (b <= 0x7f800000u && b > m) m = b;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = max(m, red[w]);
+    // amax = f * 2^E with f in [0.5, 1); 448 = 0.875 * 2^9, so e = E - 9 if f <= 0.875, else E - 8
+    int e = 0;
+    if (m != 0u && m < 0x7f800000u) {
+        const float amax = __uint_as_float(m);
+        int E;
+        const float f = frexpf(amax, &E);
+        e = (f <= 0.875f) ? E - 9 : E - 8;
+        e = max(-127, min(127, e));
+    }
+    const float down = exp2f((float)-e), up = exp2f((float)e);
+    if (threadIdx.x == 0) scales[row] = up;
+    uint2 *dst = reinterpret_cast<uint2 *>(codes + row * n_in);
+    uint4 *dq = dequant ? reinterpret_cast<uint4 *>(dequant + row * n_in) : nullptr;
+    for (int i = threadIdx.x; i < n8; i += 256) {
+        const uint4 v = src[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t c[4];   // two codes each (low 16 bits)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint16_t pair;
+            const float lo = bf16_lo(w[k]) * down, hi = bf16_hi(w[k]) * down;
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(hi), "f"(lo));
+            c[k] = pair;
+        }
+        dst[i] = make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+        if (dq) {
+            uint32_t o[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                uint32_t h2;
+                asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)c[k]));
+                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+                o[k] = pack_bf16x2(f.x * up, f.y * up);   // at most 4 significant bits times a power of two: exact
+            }
+            dq[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_quantise_rows_e4m3(const LaunchCtx &lc, const bf16 *W, uint8_t *codes, float *scales, bf16 *dequant,
+                                      int n_out, int n_in) {
+    if (n_out <= 0 || n_in <= 0 || n_in % 8) return cudaErrorInvalidValue;
+    LaunchCtx plain = lc;
+    plain.pdl = false;
+    return launch(plain, quantise_rows_e4m3_kernel, dim3((unsigned)n_out), dim3(256), W, codes, scales, dequant, n_in);
+}
 
 // dst (fp16 bits) = src (bf16) * 2^e; scales: DEVICE float[2] receiving {2^e, 2^-e}; max_bits: DEVICE scratch word.
 // Stream-ordered, no host synchronisation.

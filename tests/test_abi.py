@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(binding):
 def _cfg(binding, **kw):
     base = dict(n_layers=36, hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, intermediate=12288, vocab=151936,
                 max_seq=4352, max_batch=1, max_tokens=1, tie_embeddings=0, rms_eps=1e-6, rope_theta=1e6,
-                fast_bf16_activations=0)
+                tc_operands=0, serial_launches=0)
     base.update(kw)
     return binding.nnc_config(**base)
 
@@ -51,10 +51,15 @@ def test_workspace_bytes_is_host_arithmetic(binding):
     assert n2 - n >= kv
     tied = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, tie_embeddings=1)))
     assert n - tied == 151936 * 4096 * 2
+    # prompt-phase capacity beyond 128 tokens adds the fp16 copies of Wo, Wgate/up, Wdown in operand mode 0 only
+    big0 = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, max_tokens=8192)))
+    big1 = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, max_tokens=8192, tc_operands=1)))
+    assert big0 - big1 == 2 * 36 * (4096 * 4096 + 3 * 12288 * 4096)
 
 
 @pytest.mark.parametrize("bad", [dict(head_dim=64), dict(n_q_heads=30), dict(hidden=1000), dict(max_seq=0),
-                                 dict(n_kv_heads=2), dict(max_tokens=0), dict(rms_eps=0.0), dict(vocab=-1)])
+                                 dict(n_kv_heads=2), dict(max_tokens=0), dict(rms_eps=0.0), dict(vocab=-1),
+                                 dict(tc_operands=3)])
 def test_invalid_configs_are_rejected(binding, bad):
     assert binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, **bad))) == 0
 

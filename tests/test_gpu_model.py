@@ -100,6 +100,34 @@ def test_tiny_model_prefill_then_decode(oracle_mod, name, seed, gains):
     assert m.device_status() == 0
 
 
+@pytest.mark.parametrize("tc_operands", [0, 1])
+def test_tiny_model_prompt_of_more_than_128_tokens(oracle_mod, tc_operands):
+    """Calls of more than 128 tokens take the prompt-phase form of the GEMMs (tokens on the 128-row side).  Operand
+    mode 0 feeds O, gate/up and down with one fp16 term from the fp16 weight copies, mode 1 feeds two bf16 terms
+    everywhere; both must match the oracle at every position, and a second call continues from the cache."""
+    from paper_2512_21571_b200 import binding
+    from gpu_util import to_cpu
+    shape = synth.SHAPES["tiny-untied"]
+    P1, P2 = 150, 131
+    w = synth.make_weights(shape, 41, device="cuda", sigma=0.05)
+    synth.random_gains(w, 42)
+    m = binding.Model(shape, w, max_seq=P1 + P2, max_tokens=P1, tc_operands=tc_operands)
+    o = oracle_mod.Oracle(shape, to_cpu(w), max_seq=P1 + P2)
+    toks = synth.prompt_tokens(shape, 41, P1 + P2)
+    for part, n in ((toks[:P1], P1), (toks[P1:], P2)):
+        taps = torch.zeros(shape.n_layers + 1, n, shape.hidden, device="cuda")
+        m.set_hidden_tap(taps)
+        lg = m.prefill(part.cuda().view(1, n).contiguous(), all_positions=True)
+        lo, to = o.forward(part, all_positions=True, want_taps=True)
+        assert rel_l2(taps, to) < HID_TOL
+        assert (lg[0].cpu() - lo).abs().max().item() < LOGIT_TOL
+    for l in range(shape.n_layers):
+        kg, vg = m.kv_export(l, 0, P1 + P2)
+        ko, vo = o.kv_export(l, P1 + P2)
+        assert rel_l2(kg, ko) < HID_TOL and rel_l2(vg, vo) < HID_TOL, l
+    assert m.device_status() == 0
+
+
 def test_graph_equals_kernel_by_kernel_and_is_deterministic(oracle_mod):
     shape = synth.SHAPES["tiny-untied"]
     m, o, w = make_pair(oracle_mod, shape, 7, max_seq=64, max_tokens=8)
@@ -133,7 +161,7 @@ def test_prefill_equals_stepwise_decode_on_gpu(oracle_mod):
     logits = torch.empty(shape.vocab, device="cuda")
     for i in range(12):
         m.decode_step(toks[i:i + 1].contiguous(), logits)
-        assert (logits - la[i]).abs().max().item() < LOGIT_TOL, i
+        assert (logits - la[i]).abs().max().item() < LOGIT_TOL / 2, i
     # split prefill: 5 tokens, then 7 (positions continue from the cache length)
     m.set_length(0)
     m.prefill(toks[:5].contiguous().view(1, 5), want_logits=False)

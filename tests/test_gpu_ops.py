@@ -176,6 +176,48 @@ def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
     assert torch.allclose(Yb.float(), ref.float(), rtol=2e-2, atol=2e-2)
 
 
+def test_f16_scaled_weight_copy_is_exact(nnc):
+    """The fp16 copy holds W * 2^e exactly: dividing by the scale gives the bf16 values back, bit for bit -- also for
+    a matrix whose columns are spread over 12 more binades and for one with a large outlier."""
+    W = _w(31, 1, (512, 256))
+    for case in range(3):
+        M = W.clone()
+        if case == 1:
+            M[3, 5] = 96.0                                   # an outlier sets the scale
+        if case == 2:
+            M = (M.float() * torch.exp2(-torch.arange(256, device="cuda").float() % 12)).to(torch.bfloat16)
+        h, scales = nnc.op_to_f16_scaled(M)
+        torch.cuda.synchronize()
+        sc, inv = scales.tolist()
+        assert sc * inv == 1.0 and math.log2(sc) == int(math.log2(sc))
+        amax = M.float().abs().max().item() * sc
+        assert 2.0 ** 14 <= amax < 2.0 ** 15
+        assert torch.equal(h.float() * inv, M.float())
+
+
+@pytest.mark.parametrize("T,N,K", [(129, 256, 64), (300, 1000, 384), (1024, 512, 1024), (515, 264, 2048)])
+def test_gemm_f16_against_oracle(nnc, oracle_mod, T, N, K):
+    """One-term fp16 GEMM (the prompt-phase form): fp16 activations, scaled fp16 weight copy, scale undone in the
+    epilogue.  The oracle multiplies the same values (fp16 activations are exact in fp32, weights are bf16)."""
+    W = _w(32, 1, (N, K))
+    X = synth.normal(32, 2, (T, K), 1.0, torch.float32, "cuda").to(torch.float16)
+    W16, scales = nnc.op_to_f16_scaled(W)
+    want = oracle_mod.matmul(W.cpu(), X.float().cpu())
+    Y = nnc.op_gemm_f16(X, W16, out_scale=scales[1:])
+    assert nnc.op_status() == 0
+    assert torch.allclose(Y.cpu(), want, rtol=1e-4, atol=2e-5 * math.sqrt(K))
+    acc = synth.normal(32, 3, (T, N), 1.0, torch.float32, "cuda")
+    Y2 = nnc.op_gemm_f16(X, W16, out_scale=scales[1:], accumulate_into=acc.clone())
+    assert torch.allclose(Y2.cpu(), acc.cpu() + want, rtol=1e-4, atol=2e-5 * math.sqrt(K))
+    if N % 16 == 0:
+        A = nnc.op_gemm_swiglu_f16(X, W16, out_scale=scales[1:])
+        g, u = want[:, 0::2].double(), want[:, 1::2].double()
+        ref = g / (1 + torch.exp(-g)) * u
+        # one fp16 rounding of the result (2^-11 relative) on top of the fp32 accumulation noise
+        assert torch.allclose(A.double().cpu(), ref, rtol=1e-3, atol=1e-4 * math.sqrt(K) * 0.02 + 1e-6)
+    assert nnc.op_status() == 0
+
+
 @pytest.mark.parametrize("batch,T,nq,nkv,n_past,growth", [
     (1, 19, 2, 1, 0, 0.0), (2, 130, 4, 2, 7, 0.0), (1, 300, 8, 2, 0, 0.0), (1, 64, 16, 8, 200, 0.0),
     (1, 128, 1, 1, 0, 0.0), (1, 129, 2, 2, 127, 0.0),            # exactly one tile; one row past a tile boundary
