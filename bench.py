@@ -45,6 +45,8 @@ WORKLOADS = {
     "qwen3-8b-decode-b1-ctx4096": dict(shape="qwen3-8b", kind="decode", ctx=4096, pass_steps=128, batch=1, seed=3),
     "qwen3-1.7b-decode-b1-ctx512": dict(shape="qwen3-1.7b", kind="decode", ctx=512, pass_steps=256, batch=1, seed=2),
     "qwen3-0.6b-decode-b1-ctx64": dict(shape="qwen3-0.6b", kind="decode", ctx=64, pass_steps=64, batch=1, seed=1),
+    "qwen3-8b-decode-b1-ctx4096-fp8": dict(shape="qwen3-8b", kind="decode", ctx=4096, pass_steps=128, batch=1, seed=3,
+                                           weight_format=1),
     "qwen3-8b-decode-b32-ctx8192": dict(shape="qwen3-8b", kind="decode", ctx=8192, pass_steps=16, batch=32, seed=4),
     "qwen3-8b-prefill-4x2048": dict(shape="qwen3-8b", kind="prefill", ctx=0, tokens=2048, batch=4, seed=4),
     "qwen3-1.7b-prefill-1x512": dict(shape="qwen3-1.7b", kind="prefill", ctx=0, tokens=512, batch=1, seed=2),
@@ -195,7 +197,8 @@ def build_model(wl, max_tokens=None, w=None):
     else:
         max_seq = wl["tokens"]
         mt = wl["batch"] * wl["tokens"]
-    m = binding.Model(shape, w, max_seq=max_seq, max_batch=wl["batch"], max_tokens=max_tokens or mt)
+    m = binding.Model(shape, w, max_seq=max_seq, max_batch=wl["batch"], max_tokens=max_tokens or mt,
+                      weight_format=wl.get("weight_format", 0))
     if wl["ctx"]:
         for b in range(wl["batch"]):
             for l in range(shape.n_layers):
@@ -206,8 +209,12 @@ def build_model(wl, max_tokens=None, w=None):
     return m, shape, w
 
 
-def decode_bytes_per_step(shape, batch, ctx_mid):
-    return shape.weight_bytes_per_decode_step() + batch * ctx_mid * shape.kv_bytes_per_position()
+def decode_bytes_per_step(shape, batch, ctx_mid, weight_format=0):
+    wbytes = shape.weight_bytes_per_decode_step()
+    if weight_format == 1:   # FP8 codes: one byte per weight plus one fp32 scale per output row
+        rows = shape.n_layers * (shape.q_dim + 2 * shape.kv_dim + shape.hidden + 2 * shape.intermediate + shape.hidden) + shape.vocab
+        wbytes = wbytes // 2 + 4 * rows
+    return wbytes + batch * ctx_mid * shape.kv_bytes_per_position()
 
 
 def prefill_flops(shape, batch, T):
@@ -322,7 +329,7 @@ def time_prefill(m, shape, wl, steps, warmup, world, host=False):
     return ms, m.launch_count - n0, sampler.summary(), B * T * 4, B * shape.vocab * 4
 
 
-def kernel_roofline_gemv(shape, peaks, w):
+def kernel_roofline_gemv(shape, peaks, w, fp8=False):
     """The dominant decode kernel -- the fused RMSNorm + gate/up GEMV + SwiGLU -- timed alone with CUDA events
     over every layer's own matrix in turn (each larger than L2, so nothing is re-read from cache)."""
     from paper_2512_21571_b200 import binding
@@ -338,43 +345,51 @@ def kernel_roofline_gemv(shape, peaks, w):
         wgu[0::2] = lw["w_gate"]
         wgu[1::2] = lw["w_up"]
         mats.append(wgu)
+    if fp8:   # the same matrices as E4M3 codes + row scales
+        q = [binding.op_quantise_rows_e4m3(W, want_dequant=False)[:2] for W in mats]
+        mats = None
+        run = lambda i, chained: binding.op_gemv_fp8(q[i][0], q[i][1], x, mode=2, gain=gain, y=y, chained=chained)
+        n_mats = len(q)
+    else:
+        run = lambda i, chained: binding.op_gemv(mats[i], x, mode=2, gain=gain, y=y, chained=chained)
     x = synth.normal(9, 1, (H,), 1.0, torch.float32, "cuda")
     gain = torch.ones(H, dtype=torch.bfloat16, device="cuda")
     y = torch.empty(I, dtype=torch.float32, device="cuda")
-    reps = 3 if mats[0].numel() * 2 * n_mats > 4 * L2_BYTES else 1
-    for W in mats[:3]:
-        binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=True)
+    wb = 1 if fp8 else 2
+    reps = 3 if 2 * I * H * wb * n_mats > 4 * L2_BYTES else 1
+    for i in range(min(3, n_mats)):
+        run(i, True)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n = 0
     e0.record()
     for _ in range(reps):
-        for W in mats:
-            binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=True)   # launched as inside the decode graph
+        for i in range(n_mats):
+            run(i, True)   # launched as inside the decode graph
             n += 1
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / n
     # one launch at a time: plain stream order, an event pair around every launch, so no launch hides its start-up
     # under its predecessor's tail
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in mats]
-    for (a, b), W in zip(pairs, mats):
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_mats)]
+    for i, (a, b) in enumerate(pairs):
         a.record()
-        binding.op_gemv(W, x, mode=2, gain=gain, y=y, chained=False)
+        run(i, False)
         b.record()
     torch.cuda.synchronize()
     iso = sorted(a.elapsed_time(b) * 1e3 for a, b in pairs)
     us_iso = iso[len(iso) // 2]
-    nbytes = 2 * I * H * 2
+    nbytes = 2 * I * H * wb + (4 * 2 * I if fp8 else 0)
     ach = nbytes / (us * 1e-6) / 1e9
     ach_iso = nbytes / (us_iso * 1e-6) / 1e9
-    return {"bound": "hbm", "kernel": "gemv_stream_kernel<SwiGLU, norm prologue>", "shape": [2 * I, H],
+    return {"bound": "hbm", "kernel": "gemv_stream_kernel<SwiGLU, norm prologue%s>" % (", FP8 codes" if fp8 else ""), "shape": [2 * I, H],
             "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
             "peak_source": peaks["source"], "bytes_per_launch": nbytes, "us_per_launch": round(us, 2),
             "launches_timed": n, "how": "back-to-back launches with programmatic stream serialization, as in the decode graph",
             "isolated_us_per_launch": round(us_iso, 2), "isolated_achieved": round(ach_iso, 1),
             "isolated_frac": round(ach_iso / peaks["hbm_gbs"], 4),
-            "traffic": measured_traffic("gemv_stream_kernel<SwiGLU>:%dx%d" % (2 * I, H))}
+            "traffic": measured_traffic("gemv_stream_kernel<SwiGLU%s>:%dx%d" % (",fp8" if fp8 else "", 2 * I, H))}
 
 
 def kernel_roofline_gemm(shape, peaks, T):
@@ -543,7 +558,8 @@ def metric_name(wl):
 
 def config_of(wl):
     c = {"workload": None, "model_shape": wl["shape"], "batch": wl["batch"], "l2": "inputs larger than L2 (weights streamed once per step)",
-         "weights": "random init N(0, 0.02^2) bf16", "tokens": "uniform random ids"}
+         "weights": "random init N(0, 0.02^2) bf16" + (", quantised at create time to FP8 E4M3 codes with a power-of-two "
+                    "scale per output row" if wl.get("weight_format", 0) == 1 else ""), "tokens": "uniform random ids"}
     for k, v in WORKLOADS.items():
         if v is wl:
             c["workload"] = k
@@ -586,7 +602,7 @@ def main():
     if args.kernel_only:
         shape = synth.SHAPES[wl["shape"]]
         if wl["kind"] == "decode" and wl["batch"] == 1:
-            roof = kernel_roofline_gemv(shape, peaks, None)
+            roof = kernel_roofline_gemv(shape, peaks, None, fp8=wl.get("weight_format", 0) == 1)
         elif wl["kind"] == "decode":
             roof = kernel_roofline_attn(shape, peaks, wl["batch"], wl["ctx"])
         else:
@@ -603,7 +619,7 @@ def main():
         ms_e, h2d, d2h = time_decode_e2e(m, shape, wl, steps, warmup, world)
         ms_e, e2e_value = whole_job_throughput(ms_e, steps, units_per_step, world)
         ctx_mid = wl["ctx"] + min(steps, wl["pass_steps"]) / 2.0
-        nbytes = decode_bytes_per_step(shape, wl["batch"], ctx_mid)
+        nbytes = decode_bytes_per_step(shape, wl["batch"], ctx_mid, wl.get("weight_format", 0))
         ach = nbytes / (ms / steps * 1e-3) / 1e9
         step_roof = {"bound": "hbm", "bytes_per_step": int(nbytes), "achieved": round(ach, 1), "unit": "GB/s",
                      "peak": peaks["hbm_gbs"], "frac": round(ach / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],
@@ -630,7 +646,7 @@ def main():
 
     if rank == 0 and not args.no_extras:
         if wl["kind"] == "decode" and wl["batch"] == 1:
-            line["roofline"] = kernel_roofline_gemv(shape, peaks, w)
+            line["roofline"] = kernel_roofline_gemv(shape, peaks, w, fp8=wl.get("weight_format", 0) == 1)
         elif wl["kind"] == "decode":
             line["roofline"] = kernel_roofline_attn(shape, peaks, wl["batch"], wl["ctx"])
         else:

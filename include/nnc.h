@@ -125,8 +125,8 @@ int nnc_prefill(nnc_model *model, const int32_t *tokens, int32_t batch, int32_t 
 
 /* One decoding step (Section 4: throughput is measured over this stage).  tokens: int32 [batch]; each
  * sequence's token takes position len; len grows by one.  logits: fp32 [batch][vocab].  argmax: int32
- * [batch] or NULL; lowest index wins ties.  At batch 1 the whole step is one CUDA graph launch (captured on
- * first use for the given buffers and re-used while they stay the same). */
+ * [batch] or NULL (batch 1 only); lowest index wins ties.  The whole step is one CUDA graph launch, captured on
+ * first use for the given buffers and batch size and re-used while they stay the same. */
 int nnc_decode_step(nnc_model *model, const int32_t *tokens, int32_t batch, float *logits, int32_t *argmax);
 
 /* End-to-end variants with HOST buffers: copy the tokens to the device, run the step, copy logits (and the
@@ -170,6 +170,15 @@ int nnc_device_status(nnc_model *model, int32_t *status_out /* HOST */);
 /* Number of kernels this library launched on behalf of `model` since creation (graph nodes count once per
  * graph launch). */
 int64_t nnc_launch_count(const nnc_model *model);
+
+/* Debugging aid.  A library built with -DNNC_BOUNDS_CHECK compares, inside the kernels, the indices that rest on the
+ * host's capacity checks (cache positions, matrix row ranges, scratch slots) with their extents; a miss is counted and
+ * the access skipped (no trap, no out-of-range access).  This call synchronises the device and returns the number of
+ * misses since the last call and the code of the first one (HOST pointers); in a normal build *misses_out is -1.
+ * nnc_bounds_check_selftest launches a kernel that touches no memory and, in a checked build, reports one miss with
+ * `code` (nothing in a normal build): it shows the counter at work. */
+int nnc_bounds_check_report(int32_t *misses_out, int32_t *first_code_out);
+int nnc_bounds_check_selftest(int32_t code, void *cuda_stream);
 
 const char *nnc_last_error(const nnc_model *model); /* never NULL; valid until the next call on the model */
 const char *nnc_status_string(int status);

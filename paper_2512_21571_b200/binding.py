@@ -58,6 +58,8 @@ EXPORTS = {
     "nnc_unrepack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "nnc_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
     "nnc_launch_count": (C.c_int64, [C.c_void_p]),
+    "nnc_bounds_check_report": (C.c_int, [C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "nnc_bounds_check_selftest": (C.c_int, [C.c_int32, C.c_void_p]),
     "nnc_last_error": (C.c_char_p, [C.c_void_p]),
     "nnc_status_string": (C.c_char_p, [C.c_int]),
     "nnc_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -288,6 +290,13 @@ def op_gemm_swiglu_f16(X: torch.Tensor, W: torch.Tensor, out_scale: Optional[tor
                                    out_scale.data_ptr() if out_scale is not None else None, _stream_ptr()),
         "nnc_op_gemm_swiglu_f16")
     return Y
+
+
+def bounds_check_report():
+    """(misses, first code) since the last call; misses == -1 in a library built without -DNNC_BOUNDS_CHECK."""
+    n, code = C.c_int32(0), C.c_int32(0)
+    _ok(lib.nnc_bounds_check_report(C.byref(n), C.byref(code)), "nnc_bounds_check_report")
+    return n.value, code.value
 
 
 def op_status() -> int:

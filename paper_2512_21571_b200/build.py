@@ -23,12 +23,15 @@ def _deps():
     return d
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = src[:-3] + ".o"
+LIB_CHECKED = os.path.join(_HERE, "libnnc_checked.so")   # the same sources with -DNNC_BOUNDS_CHECK (debugging build)
+
+
+def _compile(src: str, verbose: bool, checked: bool = False) -> str:
+    obj = src[:-3] + (".checked.o" if checked else ".o")
     newest_dep = max(os.path.getmtime(p) for p in _deps() + [src])
     if os.path.exists(obj) and os.path.getmtime(obj) >= newest_dep:
         return obj
-    cmd = ["nvcc", *NVCC_FLAGS, "-c", src, "-o", obj]
+    cmd = ["nvcc", *NVCC_FLAGS, *(["-DNNC_BOUNDS_CHECK"] if checked else []), "-c", src, "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -40,19 +43,21 @@ def _compile(src: str, verbose: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Builds libnnc.so, or with checked=True the bounds-checked debugging build libnnc_checked.so."""
+    lib = LIB_CHECKED if checked else LIB
     if force:
         for s in sources():
-            o = s[:-3] + ".o"
+            o = s[:-3] + (".checked.o" if checked else ".o")
             if os.path.exists(o):
                 os.remove(o)
     with concurrent.futures.ThreadPoolExecutor(max_workers=8) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), sources()))
-    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
-        cmd = ["nvcc", "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static"]
+        objs = list(ex.map(lambda s: _compile(s, verbose, checked), sources()))
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < max(os.path.getmtime(o) for o in objs):
+        cmd = ["nvcc", "-shared", "-o", lib, *objs, "-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static"]
         subprocess.check_call(cmd)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

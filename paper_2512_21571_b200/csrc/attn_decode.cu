@@ -87,7 +87,8 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
     AttnParams p;
     p.q = q; p.q_row_stride = q_row_stride; p.kcache = kcache; p.vcache = vcache;
     p.out_f32 = out_f32; p.out_bf16 = out_bf16; p.out_bf16_lo = out_bf16_lo; p.out_row_stride = out_row_stride;
-    p.part = part; p.tickets = tickets; p.d_len = d_len; p.len_add = len_add;
+    p.part = part; p.part_floats = attn_decode_scratch_floats(batch, nq, n_splits);
+    p.tickets = tickets; p.d_len = d_len; p.len_add = len_add;
     p.nkv = nkv; p.max_seq = max_seq; p.n_splits = n_splits;
     p.g_q = fused ? fused->g_q : nullptr; p.g_k = fused ? fused->g_k : nullptr;
     p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;

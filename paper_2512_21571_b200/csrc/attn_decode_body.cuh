@@ -54,6 +54,7 @@ struct AttnParams {
     bf16 *out_bf16, *out_bf16_lo;
     int out_row_stride;
     float *part;
+    size_t part_floats;      // floats behind `part` (what the checked build compares the partial slots with)
     uint32_t *tickets;
     const int32_t *d_len;    // cached positions before this call (null = 0)
     int len_add;             // positions attended = *d_len + len_add
@@ -112,6 +113,7 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     const int c1 = min(c0 + chunk, n_ctx);
     const int n_active = (n_ctx + chunk - 1) / chunk;
     if (c0 >= n_ctx) return;  // whole CTA; takes no ticket (n_active counts only non-empty ranges)
+    if (!NNC_BC(n_ctx >= 1 && n_ctx <= p.max_seq, 3001)) return;   // the host checks the capacity before it launches
 
     // ---- K/V fragment loads of one block of 16 positions: K rows p0 + 8h + g8 (h = 0, 1), V rows
     //      p0 + {2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9}; rows past the range are clamped here and masked later ----
@@ -291,6 +293,9 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     attn_group_sync(bar_id);
 
     float *my_part = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits + split) * kPartStride;
+    if (n_active > 1 &&
+        !NNC_BC((((size_t)b * nq + (size_t)j * G + (G - 1)) * p.n_splits + split + 1) * kPartStride <= p.part_floats, 3002))
+        return;
     // partial for head g lives at my_part + g * n_splits * kPartStride
 #pragma unroll
     for (int g = 0; g < G; ++g) {

@@ -6,16 +6,19 @@
 // tensor memory, the softmax warps read it with tcgen05.ld, and write the probabilities back over it as the bf16
 // A operand of O += P V, which tcgen05.mma reads straight from tensor memory.
 //
-// One CTA per (128 query rows, query head, sequence), 192 threads:
+// One CTA per (128 query rows, query head, sequence), 320 threads:
 //   warp 0      TMA producer: K and V tiles of 128 cache positions (two 128B-swizzled boxes of 64 head-dimension
 //               elements each) into a two-stage shared-memory ring.  The tensor map's position extent is the number
 //               of valid cache rows, so rows past the end arrive as zeros (0 * stale bits would not be 0).
 //   warp 1      MMA issuer (one lane): S[j&1] = Q K_j^T into one of two score buffers, so the product of tile j+1
 //               runs while the softmax warps work on tile j; then O += P_j V_j with V as an MN-major operand (the
 //               cache row is [position][head dim], contraction over positions).
-//   warps 2-5   one thread per query row: load Q (fp32, already normalised and rotated), scale to log2 units and
-//               write it to shared memory in the swizzled K-major layout; per tile: scores -> mask (diagonal tiles)
-//               -> exp2 -> probabilities; finally O / l to the output.
+//   warps 2-9   softmax: two threads per query row (warps w and w + 4 share a tensor-memory lane quarter and split
+//               the 128 columns of a row between them; the row maximum crosses through shared memory).  They load Q
+//               (fp32; optionally applying the per-head RMSNorm and RoPE on the way: a thread holds the whole head, so
+//               the norm and the rotation pairs (i, i + 64) are thread-local), scale it to log2 units and write it to
+//               shared memory in the swizzled K-major layout; per tile: scores -> mask (diagonal tiles) -> exp2 ->
+//               probabilities; finally O / l to the output.
 // Q and P are fed as two bf16 terms (value + rounding residual) multiplied into the same accumulator: a single
 // bf16 term costs 2^-9 per operand, which the parity tolerance of deep models does not allow.
 // Online softmax with a lazy maximum: the running maximum m only moves (and O is rescaled in tensor memory) when a
@@ -30,7 +33,8 @@ namespace {
 
 constexpr int kQM = 128;                 // query rows per CTA
 constexpr int kKN = 128;                 // cache positions per tile
-constexpr int kPfThreads = 192;
+constexpr int kPfThreads = 320;
+constexpr int kSoftmaxThreads = 256;
 constexpr int kSlab = 128 * 128;         // bytes of a [128 rows][64 x 16 bit] swizzled slab
 constexpr int kTile = 2 * kSlab;         // [128][128] 16-bit tile = two slabs (head-dimension halves)
 constexpr int kPfSmem = 6 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   // Q hi, Q lo, 2 x (K, V)
@@ -83,6 +87,19 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+// tensor-memory load of 32 columns WITHOUT the wait: several may be issued back to back before one tmem_wait_ld()
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
@@ -94,6 +111,9 @@ struct PfParams {
     int row_stride;     // floats per token row = (nq + 2 nkv) * 128
     void *out, *out_lo; // [batch * T][nq * 128]: bf16 value (+ residual, nullable), or fp16
     int T, n_past, nq, nkv;
+    const bf16 *g_q;    // not null: the queries are raw projections; apply RMSNorm (this gain) and RoPE while loading
+    const float *rope;  // [max_seq][64][2] (cos, sin), read when g_q is set
+    float eps;
     int *status;
 };
 
@@ -115,6 +135,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
     auto pv_done = [&](int s) { return bars + 8u * (9 + s); };
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ float xch[2][2][kQM];   // [tile parity][column half][row]: the pair's half-row maxima (and, at the end, sums)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
@@ -128,10 +149,10 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
 
     if (threadIdx.x == 0) {
         abort_s = 0;
-        mbar_init(q_ready, 128);
+        mbar_init(q_ready, kSoftmaxThreads);
         for (int s = 0; s < 2; ++s) {
             mbar_init(k_full(s), 1); mbar_init(v_full(s), 1); mbar_init(s_full(s), 1);
-            mbar_init(p_full(s), 128); mbar_init(pv_done(s), 1);
+            mbar_init(p_full(s), kSoftmaxThreads); mbar_init(pv_done(s), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -202,80 +223,120 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 umma_commit(pv_done(s));
             }
         }
-    } else {   // ---------------- softmax warps 2..5: one thread per query row ----------------
+    } else {   // ---------------- softmax warps 2..9: two threads per query row ----------------
         const int quarter = warp & 3;                    // the TMEM lane quarter this warp may touch
+        const int half = (warp - 2) >> 2;                // which 64 of a row's 128 columns this thread owns
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int tok = q0 + r;
         const bool valid = tok < p.T;
         const int pos = p.n_past + tok;                  // absolute position of this row's query
+        // the two warps of a quarter meet on their own named barrier (ids 2..5)
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory"); };
         pdl_wait();
-        {   // Q -> shared memory, K-major with the 128-byte swizzle (16-byte chunk index XOR row % 8), value + residual
+        {   // Q -> shared memory, K-major with the 128-byte swizzle (16-byte chunk index XOR row % 8), value + residual.
+            // Both threads of a row read the whole head (the norm and the rotation need all of it) and each writes the
+            // eight 16-byte chunks of its own half.
             const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
             const float *src = p.qkv + ((size_t)seq * p.T + (size_t)min(tok, p.T - 1)) * p.row_stride + (size_t)h * kHeadDim;
+            float q[128];
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                float4 a = reinterpret_cast<const float4 *>(src)[2 * c], b = reinterpret_cast<const float4 *>(src)[2 * c + 1];
-                if (!valid) { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
-                const float f[8] = {a.x * qscale, a.y * qscale, a.z * qscale, a.w * qscale,
-                                    b.x * qscale, b.y * qscale, b.z * qscale, b.w * qscale};
+            for (int c = 0; c < 32; ++c) {
+                const float4 a = reinterpret_cast<const float4 *>(src)[c];
+                q[4 * c] = a.x; q[4 * c + 1] = a.y; q[4 * c + 2] = a.z; q[4 * c + 3] = a.w;
+            }
+            if (p.g_q) {
+                float ss = 0.f;
+#pragma unroll
+                for (int e = 0; e < 128; ++e) ss = fmaf(q[e], q[e], ss);
+                const float inv = rsqrtf(ss * (1.f / kHeadDim) + p.eps);
+                const float *cs = p.rope + (size_t)min(pos, p.n_past + p.T - 1) * kHeadDim;   // (cos, sin) of pair i at 2i
+#pragma unroll
+                for (int i = 0; i < 64; i += 2) {
+                    const float4 t = *reinterpret_cast<const float4 *>(cs + 2 * i);         // c_i s_i c_{i+1} s_{i+1}
+                    const uint32_t ga = *reinterpret_cast<const uint32_t *>(p.g_q + i), gb = *reinterpret_cast<const uint32_t *>(p.g_q + 64 + i);
+                    const float a0 = q[i] * inv * bf16_lo(ga), a1 = q[i + 1] * inv * bf16_hi(ga);
+                    const float b0 = q[64 + i] * inv * bf16_lo(gb), b1 = q[65 + i] * inv * bf16_hi(gb);
+                    q[i] = a0 * t.x - b0 * t.y;      q[i + 1] = a1 * t.z - b1 * t.w;
+                    q[64 + i] = b0 * t.x + a0 * t.y; q[65 + i] = b1 * t.z + a1 * t.w;
+                }
+            }
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e)   // compile-time indices on both sides keep q[] in registers; half is warp-uniform
+                    f[e] = valid ? (half ? q[64 + 8 * cc + e] : q[8 * cc + e]) * qscale : 0.f;
                 uint4 hi, lo;
                 hi.x = pack_bf16x2(f[0], f[1]); lo.x = pack_bf16x2(f[0] - bf16_lo(hi.x), f[1] - bf16_hi(hi.x));
                 hi.y = pack_bf16x2(f[2], f[3]); lo.y = pack_bf16x2(f[2] - bf16_lo(hi.y), f[3] - bf16_hi(hi.y));
                 hi.z = pack_bf16x2(f[4], f[5]); lo.z = pack_bf16x2(f[4] - bf16_lo(hi.z), f[5] - bf16_hi(hi.z));
                 hi.w = pack_bf16x2(f[6], f[7]); lo.w = pack_bf16x2(f[6] - bf16_lo(hi.w), f[7] - bf16_hi(hi.w));
-                const uint32_t off = (uint32_t)(c >> 3) * kSlab + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                const uint32_t off = (uint32_t)half * kSlab + (uint32_t)r * 128u + (uint32_t)((cc ^ (r & 7)) << 4);
                 sts128(q_hi + off, hi);
                 sts128(q_lo + off, lo);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes, async-proxy (MMA) reads
             mbar_arrive(q_ready);
         }
-        float m_used = -INFINITY, l = 0.f;
-        bool ok = true;
+        float m_used = -INFINITY, l = 0.f;   // l: this thread's share of the row sum
+        // A warp whose wait ran out goes `dead`: it touches nothing any more but keeps meeting its partner at every
+        // pair barrier (one per tile and one at the end), so the partner can never be left waiting at one.
+        bool dead = false;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1, u = j >> 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(s_full(s), (uint32_t)(u & 1), abort_flag, p.status, 27));
-            if (!ok) break;
-            tc_fence_after();
+            if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(s_full(s), (uint32_t)(u & 1), abort_flag, p.status, 27));
             const uint32_t ts = tmem_base + lane_addr + kColS + (uint32_t)s * kKN;
-            float sv[128];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t t[32];
-                tmem_ld32(ts + 32u * i, t);
-#pragma unroll
-                for (int e = 0; e < 32; ++e) sv[32 * i + e] = __uint_as_float(t[e]);
-            }
-            const int k0 = j * kKN;
-            if (k0 + kKN - 1 > p.n_past + q0) {   // the tile reaches past the first row's position: causal mask
-#pragma unroll
-                for (int e = 0; e < 128; ++e)
-                    if (k0 + e > pos) sv[e] = -INFINITY;
-            }
+            float sv[64];
             float m_tile = -INFINITY;
+            if (!dead) {
+                tc_fence_after();
+                uint32_t t0[32], t1[32];
+                tmem_ld32_nowait(ts + 64u * half, t0);
+                tmem_ld32_nowait(ts + 64u * half + 32u, t1);
+                tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 128; ++e) m_tile = fmaxf(m_tile, sv[e]);
+                for (int e = 0; e < 32; ++e) { sv[e] = __uint_as_float(t0[e]); sv[32 + e] = __uint_as_float(t1[e]); }
+                const int k0 = j * kKN + 64 * half;   // cache position of this thread's first column
+                if (j * kKN + kKN - 1 > p.n_past + q0) {   // the tile reaches past the first row's position: causal mask
+#pragma unroll
+                    for (int e = 0; e < 64; ++e)
+                        if (k0 + e > pos) sv[e] = -INFINITY;
+                }
+#pragma unroll
+                for (int e = 0; e < 64; ++e) m_tile = fmaxf(m_tile, sv[e]);
+                xch[s][half][r] = m_tile;
+            }
+            // After this barrier both threads of a row hold their scores in registers, so the probability columns may
+            // be written over the partner's score columns (value pairs of positions 64..127 land in columns 32..63,
+            // residual pairs of positions 0..63 in columns 64..95).
+            pair_sync();
+            if (dead) continue;
+            m_tile = fmaxf(m_tile, xch[s][half ^ 1][r]);
             if (j == 0) {
                 m_used = m_tile;   // finite: position 0 is visible to every row
             } else {
-                const bool need = m_tile > m_used + kLazyMax;
+                const bool need = m_tile > m_used + kLazyMax;   // the same verdict in both threads of the row
                 if (__any_sync(0xffffffffu, need)) {
-                    // O is rescaled in tensor memory; the product of the previous tile must have landed first
-                    ok = __all_sync(0xffffffffu, mbar_wait(pv_done((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, p.status, 28));
-                    if (!ok) break;
+                    // O is rescaled in tensor memory (each thread its 64 columns); the product of the previous tile
+                    // must have landed first
+                    dead = !__all_sync(0xffffffffu, mbar_wait(pv_done((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, p.status, 28));
+                    if (dead) continue;
                     tc_fence_after();
                     const float m_new = need ? m_tile : m_used;
                     const float alpha = exp2f(m_used - m_new);   // 1 for the rows that keep their maximum
-                    const uint32_t to = tmem_base + lane_addr + kColO;
-#pragma unroll 1
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t t[32];
-                        tmem_ld32(to + 32u * i, t);
+                    const uint32_t to = tmem_base + lane_addr + kColO + 64u * half;
+                    uint32_t t0[32], t1[32];
+                    tmem_ld32_nowait(to, t0);
+                    tmem_ld32_nowait(to + 32u, t1);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) t[e] = __float_as_uint(__uint_as_float(t[e]) * alpha);
-                        tmem_st32(to + 32u * i, t);
+                    for (int e = 0; e < 32; ++e) {
+                        t0[e] = __float_as_uint(__uint_as_float(t0[e]) * alpha);
+                        t1[e] = __float_as_uint(__uint_as_float(t1[e]) * alpha);
                     }
+                    tmem_st32(to, t0);
+                    tmem_st32(to + 32u, t1);
                     tmem_wait_st();
                     l *= alpha;
                     m_used = m_new;
@@ -283,11 +344,12 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
             }
             float sum = 0.f;
 #pragma unroll
-            for (int e = 0; e < 128; ++e) { sv[e] = exp2f(sv[e] - m_used); sum += sv[e]; }
+            for (int e = 0; e < 64; ++e) { sv[e] = exp2f(sv[e] - m_used); sum += sv[e]; }
             l += sum;
-            // P over S: value pairs in columns 0..63, residual pairs in columns 64..127 (two positions per column)
+            // P over S: value pairs in columns 0..63, residual pairs in columns 64..127 (two positions per column);
+            // this thread's 64 positions are columns 32 * half .. + 31 of each
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 2; ++i) {
                 uint32_t ph[16], pl[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
@@ -295,22 +357,25 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                     ph[e] = pack_bf16x2(a, b);
                     pl[e] = pack_bf16x2(a - bf16_lo(ph[e]), b - bf16_hi(ph[e]));
                 }
-                tmem_st16(ts + 16u * i, ph);
-                tmem_st16(ts + 64u + 16u * i, pl);
+                tmem_st16(ts + 32u * half + 16u * i, ph);
+                tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(p_full(s));
         }
-        // ---- O / l -> output ----
+        bool ok = !dead;
+        // ---- O / l -> output: the pair adds its partial row sums, each thread writes its 64 columns ----
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done((n_tiles - 1) & 1), (uint32_t)(((n_tiles - 1) >> 1) & 1), abort_flag, p.status, 29));
+        xch[n_tiles & 1][half][r] = l;   // the parity the last tile did not use
+        pair_sync();
         if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l;
-            const uint32_t to = tmem_base + lane_addr + kColO;
-            const size_t oi = ((size_t)seq * p.T + (size_t)tok) * p.nq * kHeadDim + (size_t)h * kHeadDim;
+            const float inv = 1.f / (l + xch[n_tiles & 1][half ^ 1][r]);
+            const uint32_t to = tmem_base + lane_addr + kColO + 64u * half;
+            const size_t oi = ((size_t)seq * p.T + (size_t)tok) * p.nq * kHeadDim + (size_t)h * kHeadDim + 64 * half;
 #pragma unroll 1
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 2; ++i) {
                 uint32_t t[32];
                 tmem_ld32(to + 32u * i, t);
                 if (!valid) continue;
@@ -397,7 +462,7 @@ cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensor
 // sequence s; the cache must already hold their K/V.  n_past is a host value: it sizes the tensor maps.
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
                                 const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
-                                int n_past) {
+                                int n_past, const AttnFused *fused) {
     const int batch = rows / rows_per_seq, T = rows_per_seq;
     if (T <= 0 || batch <= 0 || n_past < 0 || n_past + T > max_seq || nq % nkv) return cudaErrorInvalidValue;
     if (((uintptr_t)qkv | (uintptr_t)kcache | (uintptr_t)vcache | (uintptr_t)out | (uintptr_t)out_lo) & 15) return cudaErrorInvalidValue;
@@ -407,6 +472,7 @@ cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows,
     PfParams p;
     p.qkv = qkv; p.row_stride = (nq + 2 * nkv) * kHeadDim; p.out = out; p.out_lo = out_lo;
     p.T = T; p.n_past = n_past; p.nq = nq; p.nkv = nkv; p.status = lc.status;
+    p.g_q = fused ? fused->g_q : nullptr; p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;
     const dim3 grid((T + kQM - 1) / kQM, nq, batch);
     return out_fp16 ? launch_pf<true>(lc, mk, mv, p, grid) : launch_pf<false>(lc, mk, mv, p, grid);
 }

@@ -56,6 +56,35 @@ __device__ __forceinline__ float warp_max(float v) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- bounds-checked debugging build (-DNNC_BOUNDS_CHECK) -------------------------------------------------
+// The normal library trusts the extents its launchers computed.  The checked build compares the indices that rest
+// on such an assumption (a cache position against the cache capacity, a row range against the matrix, a scratch
+// slot against the scratch size) with the extent at the point of use: a miss is COUNTED in a device word and the
+// access is skipped -- never a trap, never an out-of-range access -- and nnc_bounds_check_report() reads the count
+// and the code of the first miss.  NNC_BC(cond, code) evaluates to `cond` in the checked build and to `true` in the
+// normal one, so it wraps only conditions the normal build does not need; guards that are part of a kernel's logic
+// stay ordinary `if`s.  Each translation unit holds its own counter (no relocatable device code) and registers a
+// reader for it.
+#ifdef NNC_BOUNDS_CHECK
+static __device__ unsigned g_bc_words[2];   // {misses, code of the first miss}
+void bc_register(void (*read_and_clear)(unsigned *misses, unsigned *first_code));
+static void bc_read_this_tu(unsigned *misses, unsigned *first_code) {
+    unsigned w[2] = {0, 0}, zero[2] = {0, 0};
+    cudaMemcpyFromSymbol(w, g_bc_words, sizeof(w));
+    cudaMemcpyToSymbol(g_bc_words, zero, sizeof(zero));
+    *misses = w[0];
+    *first_code = w[1];
+}
+namespace { struct BcRegistrar { BcRegistrar() { bc_register(&bc_read_this_tu); } } g_bc_registrar; }
+__device__ __forceinline__ bool bc_check(bool ok, unsigned code) {
+    if (!ok && atomicAdd(&g_bc_words[0], 1u) == 0u) g_bc_words[1] = code;
+    return ok;
+}
+#define NNC_BC(cond, code) ::nnc::bc_check((cond), (code))
+#else
+#define NNC_BC(cond, code) true
+#endif
+
 // ---- per-CTA timeline records (tracing builds only: -DNNC_TRACE) -----------------------------------------
 // Every CTA appends {kernel id, block, SM, start, end} (globaltimer ns) to a device buffer when it exits;
 // nnc_trace_dump() copies the buffer to the host.  Compiled out of the normal library.  Each translation unit

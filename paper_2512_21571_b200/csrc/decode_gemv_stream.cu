@@ -204,8 +204,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamPa
                     const int row0 = s * p.rps;
                     const int rows = min(p.rps, p.n_out - row0);
                     slot_row[stage] = row0;
-                    bulk_load(smem_u32(ring) + (uint32_t)stage * stage_bytes, p.W + (size_t)row0 * row_bytes,
-                              (uint32_t)rows * row_bytes, smem_u32(&full[stage]));
+                    // a stage lies inside the matrix and inside its ring slot (checked build; a miss skips the copy and
+                    // the consumers' bounded wait reports it)
+                    if (NNC_BC(row0 >= 0 && rows > 0 && row0 + rows <= p.n_out && (uint32_t)rows * row_bytes <= stage_bytes &&
+                               (uint32_t)(stage + 1) * stage_bytes <= (uint32_t)kRingBytes, 1001))
+                        bulk_load(smem_u32(ring) + (uint32_t)stage * stage_bytes, p.W + (size_t)row0 * row_bytes,
+                                  (uint32_t)rows * row_bytes, smem_u32(&full[stage]));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 r0 = r1; r1 = r2; r2 = r3;

@@ -28,7 +28,7 @@ __global__ void embed_kernel(const bf16 *__restrict__ E, const int32_t *__restri
 }
 
 // One warp per (row, head) of the fused QKV activation [rows][(nq + 2 nkv) * 128] (fp32).
-//   q heads: q <- RoPE_p(RMSNorm_128(q; g_q)) in place (and optionally a bf16 copy for tensor-core attention)
+//   q heads: q <- RoPE_p(RMSNorm_128(q; g_q)) in place (left alone with skip_q: the attention kernel does it itself)
 //   k heads: the same with g_k, then rounded to bf16 into the cache at position p
 //   v heads: rounded to bf16 into the cache at position p
 // p = *d_len + (row % rows_per_seq); sequence = row / rows_per_seq.  Lane l owns elements 2l, 2l+1 and their
@@ -37,19 +37,21 @@ __global__ void __launch_bounds__(128)
 qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, const bf16 *__restrict__ g_q,
                            const bf16 *__restrict__ g_k, float eps, const float *__restrict__ rope,
                            bf16 *__restrict__ kcache, bf16 *__restrict__ vcache, int nq, int nkv, int max_seq,
-                           const int32_t *__restrict__ d_len, bf16 *__restrict__ q_bf16) {
+                           const int32_t *__restrict__ d_len, int skip_q) {
     NNC_TRACE_SCOPE(2);
     pdl_wait();
     const int heads = nq + 2 * nkv;
+    const int per_row = skip_q ? 2 * nkv : heads;   // heads of a row this launch works on (the last ones)
     const int unit = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (unit < rows * heads) {
-        const int row = unit / heads, head = unit % heads;
+    if (unit < rows * per_row) {
+        const int row = unit / per_row, head = heads - per_row + unit % per_row;
         const int seq = row / rows_per_seq;
         const int pos = *d_len + (row % rows_per_seq);
         float *p = qkv + (size_t)row * heads * kHeadDim + (size_t)head * kHeadDim;
         float2 a = reinterpret_cast<float2 *>(p)[lane];        // elements 2l, 2l+1
         float2 b = reinterpret_cast<float2 *>(p + 64)[lane];   // elements 2l+64, 2l+65
+        (void)NNC_BC(pos >= 0 && pos < max_seq, 201);          // the host checks the capacity before it launches
         if (pos < max_seq) {
             if (head < nq + nkv) {
                 const bf16 *g = head < nq ? g_q : g_k;
@@ -67,11 +69,6 @@ qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, 
             if (head < nq) {
                 reinterpret_cast<float2 *>(p)[lane] = a;
                 reinterpret_cast<float2 *>(p + 64)[lane] = b;
-                if (q_bf16) {
-                    bf16 *qb = q_bf16 + ((size_t)row * nq + head) * kHeadDim;
-                    reinterpret_cast<uint32_t *>(qb)[lane] = pack_bf16x2(a.x, a.y);
-                    reinterpret_cast<uint32_t *>(qb + 64)[lane] = pack_bf16x2(b.x, b.y);
-                }
             } else {
                 const bool is_k = head < nq + nkv;
                 const int j = is_k ? head - nq : head - nq - nkv;
@@ -172,10 +169,10 @@ cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *toke
 cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
-                                       const int32_t *d_len, bf16 *q_bf16_out) {
-    const long units = (long)rows * (nq + 2 * nkv);
+                                       const int32_t *d_len, bool skip_q) {
+    const long units = (long)rows * (skip_q ? 2 * nkv : nq + 2 * nkv);
     return launch(lc, qk_norm_rope_append_kernel, dim3((unsigned)((units + 3) / 4)), dim3(128), qkv, rows,
-                  rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, q_bf16_out);
+                  rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, skip_q ? 1 : 0);
 }
 
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,

@@ -35,6 +35,7 @@ struct GemmParams {
     int stream;          // 1: the (tile, K stage) space is cut into one contiguous range per CTA (SWAP only)
     float *part;         // stream: fp32 partial tiles [CTA][first / last segment][BN / 32][8][128 rows][4]
     uint32_t *tickets;   // stream: one "piece parked" flag per partial-tile slot, zero at rest
+    size_t part_bytes;   // stream: bytes behind `part`
     const float *out_scale;   // DEVICE scalar multiplied into every accumulator before the epilogue (nullable = 1)
     int *status;
 };
@@ -332,7 +333,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (g.piece != 0) {
                     const int my_slot = it.slot_of(blockIdx.x, tile_id);
                     float *slot = p.part + (size_t)my_slot * kSlotFloats;
-                    if (got) {
+                    if (got && NNC_BC(((size_t)my_slot + 1) * kSlotFloats * sizeof(float) <= p.part_bytes, 4001)) {
 #pragma unroll 1
                         for (int c0 = 0; c0 < BN; c0 += 32) {
                             uint32_t r[32];
@@ -589,7 +590,7 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
     // Few tokens: the product is bound by streaming the weights.  Whole tiles dealt round-robin leave SMs idle in the
     // last round (or all the time, when there are fewer tiles than SMs), so the (tile, K stage) space is cut into one
     // equal contiguous range per CTA instead; tiles that straddle a cut are finished through partial tiles in scratch.
-    p.stream = 0; p.part = nullptr; p.tickets = nullptr;
+    p.stream = 0; p.part = nullptr; p.tickets = nullptr; p.part_bytes = 0;
     const int tiles = p.m_tiles * p.n_tiles;
     int grid = tiles < lc.sm_count ? tiles : lc.sm_count;
     if (SWAP && scratch && scratch->part && scratch->tickets) {
@@ -598,7 +599,7 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
         const double whole_tile_eff = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
         const size_t need = (size_t)2 * g * BN * kBM * sizeof(float);
         if (whole_tile_eff < 0.97 && need <= scratch->part_bytes && 2 * g <= scratch->n_tickets) {
-            p.stream = 1; p.part = scratch->part; p.tickets = scratch->tickets;
+            p.stream = 1; p.part = scratch->part; p.tickets = scratch->tickets; p.part_bytes = scratch->part_bytes;
             grid = g;
         }
     }

@@ -161,7 +161,7 @@ struct nnc_model {
         cudaGraphExec_t exec;
         int64_t nodes;
     };
-    std::map<std::tuple<const void *, const void *, const void *>, Graph> graphs;
+    std::map<std::tuple<const void *, const void *, const void *, int>, Graph> graphs;
     char err[512];
 
     size_t kv_layer_stride() const { return (size_t)c.max_batch * c.n_kv_heads * c.max_seq * 128; }
@@ -228,10 +228,9 @@ int decode_b1_launches(nnc_model *m, const int32_t *tokens, float *logits, int32
 }
 
 // Token-batch path: rows = batch * T tokens; T == 1 with decode attention is a batched decode step.
-int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float *logits, int all_positions) {
+int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float *logits, int all_positions, const LaunchCtx &lc) {
     const nnc_config &c = m->c;
     const int R = batch * T, H = c.hidden, I = c.intermediate, qd = m->qd(), qkvd = m->qkvd();
-    LaunchCtx lc = ctx(m, m->pdl);
     NNC_CUDA(m, launch_embed(lc, m->embed, tokens, m->xt, R, H, c.vocab, m->taps));
     const int n_splits = attn_decode_splits(m->sm_count, batch, c.n_kv_heads, c.max_seq);
     // prompt-phase calls of more than 128 tokens: attention output, MLP input and SwiGLU output travel as one fp16 term
@@ -248,9 +247,11 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
             NNC_CUDA(m, launch_attn_decode(lc, m->qkvt, qkvd, kc, vc, nullptr, m->ob, m->ob_lo, qd, m->part, m->tickets, m->d_len, 1,
                                            batch, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
         } else {
+            // K/V heads: norm, rotation, append; the query heads are normalised and rotated by the attention kernel
             NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
-                                                   c.n_kv_heads, c.max_seq, m->d_len, nullptr));
-            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, f16 ? nullptr : m->ob_lo, f16, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len));
+                                                   c.n_kv_heads, c.max_seq, m->d_len, true));
+            const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
+            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, f16 ? nullptr : m->ob_lo, f16, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len, &fused));
         }
         if (f16) {
             NNC_CUDA(m, launch_gemm(lc, m->ob, nullptr, (const bf16 *)w.wo16, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, nullptr, true, w.sc_o + 1));
@@ -461,7 +462,7 @@ int nnc_prefill(nnc_model *m, const int32_t *tokens, int32_t batch, int32_t n_to
     if (!m || !tokens) return fail(m, NNC_ERR_INVALID_ARG, "null argument");
     int rc = check_step(m, batch, n_tokens);
     if (rc) return rc;
-    rc = forward_tokens(m, tokens, batch, n_tokens, logits, all_positions);
+    rc = forward_tokens(m, tokens, batch, n_tokens, logits, all_positions, ctx(m, m->pdl));
     if (rc == NNC_OK) m->len += n_tokens;
     return rc;
 }
@@ -470,18 +471,15 @@ int nnc_decode_step(nnc_model *m, const int32_t *tokens, int32_t batch, float *l
     if (!m || !tokens || !logits) return fail(m, NNC_ERR_INVALID_ARG, "null argument");
     int rc = check_step(m, batch, 1);
     if (rc) return rc;
-    if (batch > 1) {
-        if (argmax) return fail(m, NNC_ERR_INVALID_ARG, "argmax output is only available at batch 1");
-        rc = forward_tokens(m, tokens, batch, 1, logits, 0);
-        if (rc == NNC_OK) m->len += 1;
-        return rc;
-    }
+    if (batch > 1 && argmax) return fail(m, NNC_ERR_INVALID_ARG, "argmax output is only available at batch 1");
     if (m->taps) {  // instrumented: kernel by kernel
-        rc = decode_b1_launches(m, tokens, logits, argmax, ctx(m, false));
+        rc = batch > 1 ? forward_tokens(m, tokens, batch, 1, logits, 0, ctx(m, false))
+                       : decode_b1_launches(m, tokens, logits, argmax, ctx(m, false));
         if (rc == NNC_OK) m->len += 1;
         return rc;
     }
-    auto key = std::make_tuple((const void *)tokens, (const void *)logits, (const void *)argmax);
+    // one graph per (buffers, batch): the position is read from device memory, so a graph serves every step
+    auto key = std::make_tuple((const void *)tokens, (const void *)logits, (const void *)argmax, (int)batch);
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         // capture the step once for this set of buffers
@@ -491,7 +489,7 @@ int nnc_decode_step(nnc_model *m, const int32_t *tokens, int32_t batch, float *l
         NNC_CUDA(m, cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeThreadLocal));
         LaunchCtx cap = ctx(m, m->pdl);
         cap.stream = m->capture_stream;
-        rc = decode_b1_launches(m, tokens, logits, argmax, cap);
+        rc = batch > 1 ? forward_tokens(m, tokens, batch, 1, logits, 0, cap) : decode_b1_launches(m, tokens, logits, argmax, cap);
         cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
         const int64_t nodes = m->launches - before;
         m->launches = before;
@@ -651,6 +649,38 @@ const char *nnc_status_string(int status) {
     return "unknown status";
 }
 
+#ifdef NNC_BOUNDS_CHECK
+}  // extern "C"
+namespace nnc {
+static std::vector<void (*)(unsigned *, unsigned *)> &bc_readers() {
+    static std::vector<void (*)(unsigned *, unsigned *)> v;
+    return v;
+}
+void bc_register(void (*read_and_clear)(unsigned *, unsigned *)) { bc_readers().push_back(read_and_clear); }
+}  // namespace nnc
+extern "C" {
+#endif
+
+int nnc_bounds_check_report(int32_t *misses_out, int32_t *first_code_out) {
+    if (!misses_out || !first_code_out) return NNC_ERR_INVALID_ARG;
+#ifdef NNC_BOUNDS_CHECK
+    if (cudaDeviceSynchronize() != cudaSuccess) return NNC_ERR_CUDA;
+    unsigned total = 0, first = 0;
+    for (auto rd : nnc::bc_readers()) {
+        unsigned n = 0, code = 0;
+        rd(&n, &code);
+        if (n && !first) first = code;
+        total += n;
+    }
+    *misses_out = (int32_t)total;
+    *first_code_out = (int32_t)first;
+#else
+    *misses_out = -1;   // not a checked build
+    *first_code_out = 0;
+#endif
+    return NNC_OK;
+}
+
 #ifdef NNC_TRACE
 }  // extern "C"
 namespace nnc {
@@ -699,6 +729,12 @@ static int op_ctx(LaunchCtx &lc, void *stream) {
     if (cudaGetSymbolAddress((void **)&status, g_op_status) != cudaSuccess) return NNC_ERR_CUDA;
     lc = LaunchCtx{(cudaStream_t)stream, sms, false, nullptr, status};
     return NNC_OK;
+}
+
+int nnc_bounds_check_selftest(int32_t code, void *cuda_stream) {
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    return launch_bounds_check_selftest(lc, code) == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 
 int nnc_op_gemm(const void *X, const void *X_lo, const void *W, void *Y, int32_t T, int32_t n_out, int32_t n_in,

@@ -81,10 +81,11 @@ cudaError_t launch_quantise_rows_e4m3(const LaunchCtx &lc, const bf16 *W, uint8_
 // ---- row-wise kernels (decode_misc.cu) ----------------------------------------------------------------
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
                          int vocab, float *tap);
+// skip_q: only the key and value heads are processed (the consumer of the queries normalises and rotates them itself)
 cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
-                                       const int32_t *d_len, bf16 *q_bf16_out);
+                                       const int32_t *d_len, bool skip_q);
 // out_f16: `out` receives one fp16 matrix (saturating) instead of a bf16 value (+ residual in out_lo)
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
                                 int H, float eps, int first, int step, bool out_f16 = false);
@@ -109,9 +110,11 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
                                int max_seq, int n_splits, const AttnFused *fused);
 // prompt-phase causal attention on the tcgen05 path (attn_prefill_tc.cu); out: bf16 value (+ residual in out_lo, nullable)
 // or, with out_fp16, one fp16 matrix.  n_past (cached positions before this call) is a host value: it sizes the tensor maps.
+// fused != null: the query heads of qkv are raw projections and the kernel applies the per-head RMSNorm (g_q) and RoPE
+// itself (the K/V rows must already be in the cache: launch_qk_norm_rope_append with skip_q).
 cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
                                 const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
-                                int n_past);
+                                int n_past, const AttnFused *fused = nullptr);
 
 // ---- GEMM (gemm_tc.cu) --------------------------------------------------------------------------------
 enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwigluBf16 = 3 };
@@ -138,6 +141,8 @@ cudaError_t launch_gemm(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, co
 // dst rows [row0, row0 + rows) <- src rows [0, rows), row length K (plain row copy into a taller matrix)
 cudaError_t launch_copy_rows(const LaunchCtx &lc, const bf16 *src, bf16 *dst, int rows, int K, int dst_row0,
                              int dst_row_step, int src_row0, int src_row_step);
+
+cudaError_t launch_bounds_check_selftest(const LaunchCtx &lc, int code);   // reports one miss with `code` in a checked build
 
 // fp16 copy of a bf16 matrix scaled by a power of two (see repack.cu); scales: DEVICE float[2] <- {2^e, 2^-e}
 cudaError_t launch_to_f16_scaled(const LaunchCtx &lc, const bf16 *src, void *dst, size_t n, float *scales, uint32_t *max_bits);

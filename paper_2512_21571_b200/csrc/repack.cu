@@ -17,14 +17,19 @@ namespace nnc {
 namespace {
 
 __global__ void copy_rows_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int rows, int chunks_per_row,
-                                 int dst_row0, int dst_row_step, int src_row0, int src_row_step) {
+                                 int dst_row0, int dst_row_step, int src_row0, int src_row_step, int dst_rows_total,
+                                 int src_rows_total) {
     const size_t total = (size_t)rows * chunks_per_row;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / chunks_per_row, c = i % chunks_per_row;
-        dst[((size_t)dst_row0 + r * dst_row_step) * chunks_per_row + c] =
-            src[((size_t)src_row0 + r * src_row_step) * chunks_per_row + c];
+        const size_t dr = (size_t)dst_row0 + r * dst_row_step, sr = (size_t)src_row0 + r * src_row_step;
+        if (NNC_BC(dr < (size_t)dst_rows_total && sr < (size_t)src_rows_total, 501))
+            dst[dr * chunks_per_row + c] = src[sr * chunks_per_row + c];
     }
 }
+
+// checked build only: a kernel that reports one miss and touches no memory, so that a test can see the counter work
+__global__ void bounds_check_selftest_kernel(int code) { (void)NNC_BC(code == 0, (unsigned)code); }
 
 // max |w| over a bf16 matrix as fp32 bits (non-negative floats order like their bit patterns); NaNs are skipped
 __global__ void absmax_bits_kernel(const uint4 *__restrict__ src, size_t n_chunks, uint32_t *__restrict__ max_bits) {
@@ -181,8 +186,17 @@ cudaError_t launch_copy_rows(const LaunchCtx &lc, const bf16 *src, bf16 *dst, in
     if (blocks == 0) return cudaSuccess;
     LaunchCtx plain = lc;
     plain.pdl = false;
+    // the last row touched on either side bounds the matrices from below: what the checked build compares with
+    const int dst_rows_total = dst_row0 + (rows - 1) * dst_row_step + 1, src_rows_total = src_row0 + (rows - 1) * src_row_step + 1;
     return launch(plain, copy_rows_kernel, dim3((unsigned)blocks), dim3(256), reinterpret_cast<const uint4 *>(src),
-                  reinterpret_cast<uint4 *>(dst), rows, K / 8, dst_row0, dst_row_step, src_row0, src_row_step);
+                  reinterpret_cast<uint4 *>(dst), rows, K / 8, dst_row0, dst_row_step, src_row0, src_row_step, dst_rows_total,
+                  src_rows_total);
+}
+
+cudaError_t launch_bounds_check_selftest(const LaunchCtx &lc, int code) {
+    LaunchCtx plain = lc;
+    plain.pdl = false;
+    return launch(plain, bounds_check_selftest_kernel, dim3(1), dim3(1), code);
 }
 
 }  // namespace nnc

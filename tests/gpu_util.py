@@ -32,3 +32,15 @@ def split_bf16(x: torch.Tensor):
     """fp32 -> (hi, lo) bf16 pair with hi + lo ~ x to 16 mantissa bits: test input for the two-term GEMM operand."""
     hi = x.to(torch.bfloat16)
     return hi, (x - hi.float()).to(torch.bfloat16)
+
+
+def fp8_dequantised(oracle_mod, wc: dict, tied: bool) -> dict:
+    """The weight set of the FP8 weight format as the oracle sees it: every multiplied matrix replaced by
+    dequantise(quantise(W)) under the oracle's own row rule (CPU tensors in, CPU tensors out).  A tied embedding is the
+    lm_head, so it is replaced too; an untied embedding table is only gathered from and stays as it is."""
+    dq = lambda W: oracle_mod.dequantise_rows_e4m3(*oracle_mod.quantise_rows_e4m3(W.contiguous()))
+    out = {"embed": dq(wc["embed"]) if tied else wc["embed"],
+           "lm_head": None if wc.get("lm_head") is None else dq(wc["lm_head"]), "g_final": wc["g_final"], "layers": []}
+    for lw in wc["layers"]:
+        out["layers"].append({k: (dq(v) if k.startswith("w") else v) for k, v in lw.items()})
+    return out

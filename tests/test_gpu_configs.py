@@ -105,6 +105,53 @@ def test_config4_qwen3_8b_ctx4096_decode128(oracle_mod):
     _run(oracle_mod, "qwen3-8b", 3, prefill=0, decode=STEPS or 128, kv_prefill=4096)
 
 
+def test_config4_qwen3_8b_ctx4096_decode_fp8_weight_format(oracle_mod):
+    """The HBM-roofline workload in the second weight precision (FP8 E4M3 codes, row scales): the library quantises at
+    create time, the oracle runs on the matrices dequantised under its own rule.  NNC_TEST_FP8_STEPS decode steps."""
+    from gpu_util import fp8_dequantised, to_cpu
+    from paper_2512_21571_b200 import binding
+    name, seed, ctx = "qwen3-8b", 3, 4096
+    steps = int(os.environ.get("NNC_TEST_FP8_STEPS", "12"))
+    shape = synth.SHAPES[name]
+    w = synth.make_weights(shape, seed, device="cuda")
+    m = binding.Model(shape, w, max_seq=ctx + steps + 1, weight_format=1)
+    t0 = time.time()
+    o = oracle_mod.Oracle(shape, fp8_dequantised(oracle_mod, to_cpu(w), shape.tie_embeddings), max_seq=ctx + steps + 1)
+    t_q = time.time() - t0
+    del w
+    for l in range(shape.n_layers):
+        k, v = synth.kv_fill(shape, seed + 1000, l, ctx, device="cuda")
+        m.kv_import(l, 0, k, v)
+        o.kv_import(l, k.cpu(), v.cpu())
+    m.set_length(ctx)
+    logits = torch.empty(shape.vocab, device="cuda")
+    am = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    taps1 = torch.zeros(shape.n_layers + 1, 1, shape.hidden, device="cuda")
+    tok = int(synth.prompt_tokens(shape, seed + 1000, 1)[0])
+    dh = dl = 0.0
+    checked = 0
+    for step in range(steps):
+        tok_dev.fill_(tok)
+        tapped = step % 4 == 0
+        m.set_hidden_tap(taps1 if tapped else None)
+        m.decode_step(tok_dev, logits, am)
+        l1, t1 = o.forward(torch.tensor([tok], dtype=torch.int32), want_taps=tapped)
+        if tapped:
+            dh = max(dh, rel_l2(taps1, t1))
+        dl = max(dl, (logits.cpu() - l1).abs().max().item())
+        idx, margin = oracle_mod.argmax_margin(l1)
+        if margin > MARGIN:
+            checked += 1
+            assert int(am.item()) == idx, (step, int(am.item()), idx, margin)
+        tok = idx
+    _log(f"{name} FP8 weight format, decode {steps} steps from ctx {ctx}: hidden rel-L2 max {dh:.3e}, logits max-abs {dl:.3e}, "
+         f"argmax exact on {checked}/{steps} steps with margin > {MARGIN}; oracle quantisation {t_q:.0f}s")
+    assert dh < HID_TOL and dl < LOGIT_TOL
+    assert m.device_status() == 0
+    m.close(); o.close()
+
+
 def test_config5_mode1_qwen3_8b_prefill256_full_depth(oracle_mod):
     # the 8B shape at full depth on one 256-token sequence: what 36 layers do to the error
     _run(oracle_mod, "qwen3-8b", 4, prefill=int(os.environ.get("NNC_TEST_PREFILL", "256")), decode=STEPS or 2)

@@ -128,6 +128,48 @@ def test_tiny_model_prompt_of_more_than_128_tokens(oracle_mod, tc_operands):
     assert m.device_status() == 0
 
 
+@pytest.mark.parametrize("name,seed", [("tiny", 61), ("tiny-untied", 62)])
+def test_tiny_model_in_the_fp8_weight_format(oracle_mod, name, seed):
+    """weight_format 1: the library quantises the matrices itself; the oracle runs the same forward pass on the
+    matrices dequantised under its own rule.  Prefill goes through the tensor-core path (dequantised bf16 store), the
+    decode steps stream the FP8 codes; both must match the oracle, and the stored matrices must equal the oracle's
+    dequantised ones bit for bit."""
+    from paper_2512_21571_b200 import binding
+    from gpu_util import fp8_dequantised, to_cpu
+    shape = synth.SHAPES[name]
+    P, D = 21, 7
+    w = synth.make_weights(shape, seed, device="cuda", sigma=0.05)
+    synth.random_gains(w, seed + 1)
+    m = binding.Model(shape, w, max_seq=64, max_tokens=P, weight_format=1)
+    wq = fp8_dequantised(oracle_mod, to_cpu(w), shape.tie_embeddings)
+    o = oracle_mod.Oracle(shape, wq, max_seq=64)
+    for which, n in enumerate(["wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"]):
+        assert torch.equal(m.unrepack(0, which, w["layers"][0][n]).cpu(), wq["layers"][0][n]), n
+    toks = synth.prompt_tokens(shape, seed, P)
+    taps = torch.zeros(shape.n_layers + 1, P, shape.hidden, device="cuda")
+    m.set_hidden_tap(taps)
+    lg = m.prefill(toks.cuda().view(1, P), all_positions=True)
+    lo, to = o.forward(toks, all_positions=True, want_taps=True)
+    assert rel_l2(taps, to) < HID_TOL
+    assert (lg[0].cpu() - lo).abs().max().item() < LOGIT_TOL
+    taps1 = torch.zeros(shape.n_layers + 1, 1, shape.hidden, device="cuda")
+    logits = torch.empty(shape.vocab, device="cuda")
+    am = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tok = int(lo[-1].argmax())
+    for step in range(D):
+        tok_dev.fill_(tok)
+        m.set_hidden_tap(taps1 if step < 3 else None)     # kernel by kernel first, then the captured graph
+        m.decode_step(tok_dev, logits, am)
+        l1, t1 = o.forward(torch.tensor([tok], dtype=torch.int32), want_taps=True)
+        if step < 3:
+            assert rel_l2(taps1, t1) < HID_TOL, step
+        assert (logits.cpu() - l1).abs().max().item() < LOGIT_TOL, step
+        _check_argmax(oracle_mod, int(am.item()), l1)
+        tok = int(l1.argmax())
+    assert m.device_status() == 0
+
+
 def test_graph_equals_kernel_by_kernel_and_is_deterministic(oracle_mod):
     shape = synth.SHAPES["tiny-untied"]
     m, o, w = make_pair(oracle_mod, shape, 7, max_seq=64, max_tokens=8)

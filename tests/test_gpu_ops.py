@@ -176,6 +176,60 @@ def test_gemm_split_k_for_few_tokens(nnc, oracle_mod, T, N, K):
     assert torch.allclose(Yb.float(), ref.float(), rtol=2e-2, atol=2e-2)
 
 
+def test_quantise_rows_e4m3_matches_the_oracle_bit_for_bit(nnc, oracle_mod):
+    """Codes, row exponents and dequantised values of the device quantiser equal the oracle's (integer / byte work:
+    bit-exact), on random rows and on rows that sit on the rule's edges."""
+    W = _w(51, 1, (300, 512))
+    W[0] = 0                                  # all-zero row
+    W[1, 7] = 448.0; W[2, 7] = 450.0          # a maximum that just fits / just does not
+    W[3] = W[3] * 1e-30                       # tiny row: large negative exponent
+    W[4, :16] = torch.tensor([1.0625, 1.1875, -1.0625, 2.0 ** -10, 3 * 2.0 ** -10, 7.5 * 2.0 ** -9, 1.9999, 0.0,
+                              448.0, -448.0, 224.0, 0.4375, 0.001953125, -0.001953125, 1.0, 8.0])   # ties, subnormals
+    W[5] = W[5] * 3e4                         # large row: positive exponent
+    codes, scales, dq = nnc.op_quantise_rows_e4m3(W)
+    torch.cuda.synchronize()
+    oc, oe = oracle_mod.quantise_rows_e4m3(W.cpu())
+    assert torch.equal(scales.cpu(), torch.exp2(oe.float()))
+    assert torch.equal(codes.cpu(), oc)
+    assert torch.equal(dq.cpu().view(torch.int16), oracle_mod.dequantise_rows_e4m3(oc, oe).view(torch.int16))
+    # in place: the dequantised values may overwrite the input
+    W2 = W.clone()
+    import ctypes as C
+    assert nnc.lib.nnc_op_quantise_rows_e4m3(W2.data_ptr(), codes.data_ptr(), scales.data_ptr(), W2.data_ptr(), 300, 512,
+                                             torch.cuda.current_stream().cuda_stream) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(W2, dq) and torch.equal(codes.cpu(), oc)
+
+
+@pytest.mark.parametrize("n_out,n_in", [(16, 128), (1000, 384), (4096, 1024), (6144, 4096), (4096, 12288), (2050, 640)])
+def test_gemv_fp8_against_oracle(nnc, oracle_mod, n_out, n_in):
+    """Streaming GEMV on FP8 codes with row scales = the oracle's matmul on the dequantised matrix (store, residual,
+    norm prologue); SwiGLU on interleaved rows."""
+    W = _w(52, 1, (n_out, n_in))
+    W[n_out // 2, 3] = 0.75                   # one row with an outlier: its scale differs from its neighbours'
+    x = synth.normal(52, 2, (n_in,), 1.0, torch.float32, "cuda")
+    codes, scales, dq = nnc.op_quantise_rows_e4m3(W)
+    oc, oe = oracle_mod.quantise_rows_e4m3(W.cpu())
+    D = oracle_mod.dequantise_rows_e4m3(oc, oe)
+    assert torch.equal(codes.cpu(), oc)
+    want = oracle_mod.matmul(D, x.cpu().view(1, -1))[0]
+    tol = dict(rtol=1e-4, atol=2e-5 * math.sqrt(n_in))
+    y = nnc.op_gemv_fp8(codes, scales, x, mode=0)
+    assert torch.allclose(y.cpu(), want, **tol)
+    base = synth.normal(52, 3, (n_out,), 1.0, torch.float32, "cuda")
+    y1 = nnc.op_gemv_fp8(codes, scales, x, mode=1, y=base.clone())
+    assert torch.allclose(y1.cpu(), base.cpu() + want, **tol)
+    gain = (1.0 + synth.normal(52, 4, (n_in,), 0.1, torch.float32, "cuda")).to(torch.bfloat16)
+    h = oracle_mod.rmsnorm(x.cpu(), gain.cpu(), 1e-6)
+    want_n = oracle_mod.matmul(D, h.view(1, -1))[0]
+    yn = nnc.op_gemv_fp8(codes, scales, x, mode=0, gain=gain)
+    assert torch.allclose(yn.cpu(), want_n, **tol)
+    if n_out % 2 == 0:
+        g, u = want_n[0::2].double(), want_n[1::2].double()
+        ya = nnc.op_gemv_fp8(codes, scales, x, mode=2, gain=gain)
+        assert torch.allclose(ya.double().cpu(), g / (1 + torch.exp(-g)) * u, rtol=1e-4, atol=1e-4)
+
+
 def test_f16_scaled_weight_copy_is_exact(nnc):
     """The fp16 copy holds W * 2^e exactly: dividing by the scale gives the bf16 values back, bit for bit -- also for
     a matrix whose columns are spread over 12 more binades and for one with a large outlier."""
