@@ -468,6 +468,35 @@ def kernel_roofline_attn(shape, peaks, batch, ctx):
             "launches_timed": n, "traffic": measured_traffic("attn_decode_kernel<G=%d>:b%d_ctx%d" % (nq // nkv, batch, ctx))}
 
 
+def kernel_roofline_attn_prefill(shape, peaks, batch, T):
+    """The prompt-phase attention kernel timed alone: causal attention of `batch` sequences of T new tokens (no past).
+    Model FLOPs = 4 * 128 * T (T + 1) / 2 per head; the kernel issues twice that (Q and P travel as two bf16 terms)."""
+    from paper_2512_21571_b200 import binding
+    nq, nkv = shape.n_q_heads, shape.n_kv_heads
+    qkv = synth.normal(9, 21, (batch * T, (nq + 2 * nkv) * 128), 1.0, torch.float32, "cuda")
+    kc = synth.normal(9, 22, (batch, nkv, T, 128), 1.0, torch.bfloat16, "cuda")
+    vc = synth.normal(9, 23, (batch, nkv, T, 128), 1.0, torch.bfloat16, "cuda")
+    for _ in range(3):
+        binding.op_attn_prefill(qkv, kc, vc, T, nq, 0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 10
+    e0.record()
+    for _ in range(n):
+        binding.op_attn_prefill(qkv, kc, vc, T, nq, 0)
+    e1.record()
+    torch.cuda.synchronize()
+    assert binding.op_status() == 0
+    us = e0.elapsed_time(e1) * 1e3 / n
+    flops = 4.0 * 128 * batch * nq * (T * (T + 1) / 2)
+    ach = flops / (us * 1e-6) / 1e12
+    return {"bound": "tensor", "kernel": "attn_prefill_tc_kernel", "shape": [batch, nq, T, 128], "achieved": round(ach, 1),
+            "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ach / peaks["bf16_tflops"], 4),
+            "peak_source": peaks["source"] + " (burst)", "flops_per_launch": flops, "issued_tflops": round(2 * ach, 1),
+            "us_per_launch": round(us, 1), "launches_timed": n,
+            "traffic": measured_traffic("attn_prefill_tc_kernel:b%d_T%d" % (batch, T))}
+
+
 # ---- the CPU oracle leg (reported baseline; the only place the product's bench touches oracle/) ------------
 
 def oracle_leg(wl, shape, w_gpu, steps, warmup, budget_s=25.0):
@@ -582,6 +611,8 @@ def main():
     ap.add_argument("--kernel-only", action="store_true",
                     help="time only the dominant kernel of the workload on ~2.4 GB of operands (small enough for a "
                          "multi-pass profiler capture) and print its roofline object")
+    ap.add_argument("--kernel", default="dominant", choices=["dominant", "attention"],
+                    help="with --kernel-only on a prompt-phase workload: the GEMM (dominant) or the attention kernel")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     if args.steps is None:
@@ -605,6 +636,8 @@ def main():
             roof = kernel_roofline_gemv(shape, peaks, None, fp8=wl.get("weight_format", 0) == 1)
         elif wl["kind"] == "decode":
             roof = kernel_roofline_attn(shape, peaks, wl["batch"], wl["ctx"])
+        elif args.kernel == "attention":
+            roof = kernel_roofline_attn_prefill(shape, peaks, 1, wl["tokens"])
         else:
             roof = kernel_roofline_gemm(shape, peaks, max(wl["batch"] * wl.get("tokens", 1), 32))
         print(json.dumps({"kernel_only": True, "config": config_of(wl), "roofline": roof}), flush=True)
