@@ -84,7 +84,6 @@ template <int G>
 struct AttnSmem {
     __align__(16) float qs[G][kHeadDim];             // processed queries, pre-scaled for exp2
     float comb[kAttnWarps][G][kPartStride];          // per-warp (o~, m, l); reused for the combine weights
-    float inv_l[G];
     bool is_last;
 };
 
@@ -140,6 +139,9 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     // that is appended below
     const bool early = warp < n_blocks && !(FUSED && c0 + warp * 16 + 16 >= n_ctx);
     if (early) load_block(kfa, vfa, c0 + warp * 16);
+    // ... and so is its second block, into the other register buffer
+    const bool early2 = warp + kWarps < n_blocks && !(FUSED && c0 + (warp + kWarps) * 16 + 16 >= n_ctx);
+    if (early2) load_block(kfb, vfb, c0 + (warp + kWarps) * 16);
 
     // ---- queries (and, fused, the new token's K/V row) ----
     const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);   // scores in log2 units
@@ -260,8 +262,10 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     {
         int blk = warp;
         if (blk < n_blocks && !early) load_block(kfa, vfa, c0 + blk * 16);
+        bool have_b = early2;   // the second buffer already holds (or is receiving) the block after this one
         while (blk < n_blocks) {
-            if (blk + kWarps < n_blocks) load_block(kfb, vfb, c0 + (blk + kWarps) * 16);
+            if (blk + kWarps < n_blocks && !have_b) load_block(kfb, vfb, c0 + (blk + kWarps) * 16);
+            have_b = false;
             process_block(kfa, vfa, c0 + blk * 16);
             blk += kWarps;
             if (blk >= n_blocks) break;
@@ -336,12 +340,16 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
     if (!sm.is_last) return;
     __threadfence();
     // ---- combine (last CTA of this sequence / KV head): o = sum_c 2^(m_c - M) o~_c / sum_c 2^(m_c - M) l_c.
-    //      Weights first (one warp per head, splits across lanes), then every thread folds its output element
-    //      over the splits with all loads of a batch of splits in flight at once. ----
+    //      The splits are folded in split order, whichever CTA arrived last. ----
     float (*wgt)[kAttnMaxSplits] = reinterpret_cast<float (*)[kAttnMaxSplits]>(&sm.comb[0][0][0]);   // [G][kAttnMaxSplits], reuses comb
     const float *pbase = p.part + (((size_t)b * nq + (size_t)j * G) * p.n_splits) * kPartStride;
+    // One warp per head, 4 output elements per lane.  The (m, l) words and the first batch of partial rows are all
+    // requested before anything is waited for, so the whole combine costs one memory round trip; the weights of a
+    // head are produced and consumed by the same warp (a warp barrier suffices).
+    constexpr int kBatch = 40;
     for (int g = warp; g < G; g += kWarps) {
         const float *pp = pbase + (size_t)g * p.n_splits * kPartStride;
+        const float *pv = pp + 4 * lane;
         float mv[2], lv[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -349,33 +357,29 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams &p, int split,
             mv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim) : -INFINITY;
             lv[u] = c < n_active ? __ldcg(pp + (size_t)c * kPartStride + kHeadDim + 1) : 0.f;
         }
+        float4 v[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u)
+            v[u] = (u < n_active) ? __ldcg(reinterpret_cast<const float4 *>(pv + (size_t)u * kPartStride)) : make_float4(0.f, 0.f, 0.f, 0.f);
         const float M = warp_max(fmaxf(mv[0], mv[1]));
         const float w0 = exp2f(mv[0] - M), w1 = exp2f(mv[1] - M);
         wgt[g][lane] = w0;
         wgt[g][lane + 32] = w1;
         // fixed summation order over the splits: lane partials, then the shuffle tree
-        const float L = warp_sum(fmaf(w0, lv[0], w1 * lv[1]));
-        if (lane == 0) sm.inv_l[g] = 1.f / L;
-    }
-    attn_group_sync(bar_id);
-    // one warp per head, 4 output elements per lane: 16-byte loads, a batch of splits in flight at once
-    for (int g = warp; g < G; g += kWarps) {
-        const float *pp = pbase + (size_t)g * p.n_splits * kPartStride + 4 * lane;
+        const float il = 1.f / warp_sum(fmaf(w0, lv[0], w1 * lv[1]));
+        __syncwarp();
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int cb = 0; cb < n_active; cb += 24) {
-            float4 v[24];
 #pragma unroll
-            for (int u = 0; u < 24; ++u)
-                v[u] = (cb + u < n_active) ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(cb + u) * kPartStride))
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 24; ++u) {
-                const float w = (cb + u < n_active) ? wgt[g][cb + u] : 0.f;
-                acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
-                acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
-            }
+        for (int u = 0; u < kBatch; ++u) {
+            const float w = (u < n_active) ? wgt[g][u] : 0.f;
+            acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+            acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
         }
-        const float il = sm.inv_l[g];
+        for (int c = kBatch; c < n_active; ++c) {   // split counts beyond one batch (up to kAttnMaxSplits)
+            const float4 x = __ldcg(reinterpret_cast<const float4 *>(pv + (size_t)c * kPartStride));
+            const float w = wgt[g][c];
+            acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+        }
         const float4 r = make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il);
         const size_t oi = (size_t)b * p.out_row_stride + (size_t)(j * G + g) * kHeadDim + 4 * lane;
         if (p.out_f32) *reinterpret_cast<float4 *>(p.out_f32 + oi) = r;
