@@ -12,15 +12,18 @@
 //               of valid cache rows, so rows past the end arrive as zeros (0 * stale bits would not be 0).
 //   warp 1      MMA issuer (one lane): S[j&1] = Q K_j^T into one of two score buffers, so the product of tile j+1
 //               runs while the softmax warps work on tile j; then O += P_j V_j with V as an MN-major operand (the
-//               cache row is [position][head dim], contraction over positions).
+//               cache row is [position][head dim], contraction over positions).  Q, like P, is an A operand in
+//               TENSOR memory: a 128 x 128 x 16 instruction with both operands in shared memory would read 8 KB per
+//               64 cycles, all the shared-memory bandwidth an SM has; with A in tensor memory only K or V moves.
 //   warps 2-9   softmax: two threads per query row (warps w and w + 4 share a tensor-memory lane quarter and split
 //               the 128 columns of a row between them; the row maximum crosses through shared memory).  They load Q
 //               (fp32; optionally applying the per-head RMSNorm and RoPE on the way: a thread holds the whole head, so
 //               the norm and the rotation pairs (i, i + 64) are thread-local), scale it to log2 units and write it to
-//               shared memory in the swizzled K-major layout; per tile: scores -> mask (diagonal tiles) -> exp2 ->
+//               tensor memory as value + residual bf16 pairs; per tile: scores -> mask (diagonal tiles) -> exp2 ->
 //               probabilities; finally O / l to the output.
-// Q and P are fed as two bf16 terms (value + rounding residual) multiplied into the same accumulator: a single
-// bf16 term costs 2^-9 per operand, which the parity tolerance of deep models does not allow.
+// Q and P are fed as two bf16 terms (value + residual) multiplied into the same accumulator: a single bf16 term
+// costs 2^-9 per operand, which the parity tolerance of deep models does not allow.  Q is split by rounding; P, which
+// is produced 128 x 128 values at a time on the critical path, by truncating the fp32 bit pattern twice.
 // Online softmax with a lazy maximum: the running maximum m only moves (and O is rescaled in tensor memory) when a
 // tile's maximum exceeds it by more than 2^8; probabilities then stay below 256, which fp32 sums and the bf16
 // pair hold without loss.  The result is the exact softmax whatever m is.
@@ -37,8 +40,10 @@ constexpr int kPfThreads = 320;
 constexpr int kSoftmaxThreads = 256;
 constexpr int kSlab = 128 * 128;         // bytes of a [128 rows][64 x 16 bit] swizzled slab
 constexpr int kTile = 2 * kSlab;         // [128][128] 16-bit tile = two slabs (head-dimension halves)
-constexpr int kPfSmem = 6 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   // Q hi, Q lo, 2 x (K, V)
-constexpr uint32_t kColS = 0, kColO = 256, kTmemCols = 512;
+constexpr int kPfSmem = 4 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   // 2 x (K, V)
+// tensor-memory columns: two score / probability buffers, the output accumulator, the queries (value pairs in the
+// first 64 columns, residual pairs in the next 64; two head-dimension elements per column)
+constexpr uint32_t kColS = 0, kColO = 256, kColQ = 384, kTmemCols = 512;
 constexpr float kLazyMax = 8.f;          // log2 units
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
@@ -102,10 +107,6 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
-    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
 struct PfParams {
     const float *qkv;   // [batch * T][row_stride]: query heads first
     int row_stride;     // floats per token row = (nq + 2 nkv) * 128
@@ -123,10 +124,9 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_hi = base, q_lo = base + kTile;
-    auto k_tile = [&](int s) { return base + 2u * kTile + (uint32_t)s * 2u * kTile; };
+    auto k_tile = [&](int s) { return base + (uint32_t)s * 2u * kTile; };
     auto v_tile = [&](int s) { return k_tile(s) + (uint32_t)kTile; };
-    const uint32_t bars = base + 6u * kTile;
+    const uint32_t bars = base + 4u * kTile;
     const uint32_t q_ready = bars;
     auto k_full = [&](int s) { return bars + 8u * (1 + s); };
     auto v_full = [&](int s) { return bars + 8u * (3 + s); };
@@ -189,18 +189,24 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
             constexpr uint32_t idesc_pv = make_idesc(kHeadDim, false, true);
             bool ok = mbar_wait(q_ready, 0u, abort_flag, p.status, 22);
             tc_fence_after();
+            // Descriptors differ only in their 14-bit start-address field (bytes >> 4), so every operand descriptor of
+            // the kernel is a base computed once plus a compile-time constant: the issuing thread spends a handful of
+            // instructions per tcgen05.mma, less than the 64 cycles one 128 x 128 x 16 instruction executes for.
+            const uint32_t tq = tmem_base + kColQ;
+            const uint64_t dk[2] = {make_smem_desc(k_tile(0)), make_smem_desc(k_tile(1))};
+            const uint64_t dv[2] = {make_smem_desc_mn(v_tile(0), kSlab), make_smem_desc_mn(v_tile(1), kSlab)};
             auto issue_qk = [&](int j) -> bool {
                 const int s = j & 1, u = j >> 1;
                 if (!mbar_wait(k_full(s), (uint32_t)(u & 1), abort_flag, p.status, 23)) return false;
                 if (j >= 2 && !mbar_wait(pv_done(s), (uint32_t)((u - 1) & 1), abort_flag, p.status, 24)) return false;
                 tc_fence_after();
                 const uint32_t d = tmem_base + kColS + (uint32_t)s * kKN;
+                const uint64_t b0 = dk[s];
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dimension elements per instruction
-                    const uint32_t off = (uint32_t)(ks >> 2) * kSlab + (uint32_t)(ks & 3) * 32u;
-                    const uint64_t b = make_smem_desc(k_tile(s) + off);
-                    umma_bf16(d, make_smem_desc(q_hi + off), b, idesc_qk, ks != 0);
-                    umma_bf16(d, make_smem_desc(q_lo + off), b, idesc_qk, 1u);
+                    const uint64_t off = (uint64_t)(((ks >> 2) * kSlab + (ks & 3) * 32) >> 4);
+                    umma_bf16_ts(d, tq + (uint32_t)ks * 8u, b0 + off, idesc_qk, ks != 0);
+                    umma_bf16_ts(d, tq + 64u + (uint32_t)ks * 8u, b0 + off, idesc_qk, 1u);
                 }
                 umma_commit(s_full(s));
                 return true;
@@ -209,18 +215,23 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
             for (int j = 0; ok && j < n_tiles; ++j) {
                 if (j + 1 < n_tiles && !issue_qk(j + 1)) break;
                 const int s = j & 1, u = j >> 1;
+                const unsigned long long tr0 = NNC_TRACE_NOW();
+                (void)tr0;
                 if (!mbar_wait(p_full(s), (uint32_t)(u & 1), abort_flag, p.status, 25)) break;
+                const unsigned long long tr1 = NNC_TRACE_NOW();
+                (void)tr1;
                 if (!mbar_wait(v_full(s), (uint32_t)(u & 1), abort_flag, p.status, 26)) break;
                 tc_fence_after();
                 const uint32_t d = tmem_base + kColO;
                 const uint32_t pa = tmem_base + kColS + (uint32_t)s * kKN;   // P value in columns 0..63, residual in 64..127
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 cache positions per instruction
-                    const uint64_t b = make_smem_desc_mn(v_tile(s) + (uint32_t)ks * 2048u, kSlab);
+                    const uint64_t b = dv[s] + (uint64_t)(ks * (2048 >> 4));
                     umma_bf16_ts(d, pa + (uint32_t)ks * 8u, b, idesc_pv, (j != 0) || (ks != 0));
                     umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
                 }
                 umma_commit(pv_done(s));
+                if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) NNC_TRACE_EVENT(302, tr0, tr1, NNC_TRACE_NOW());
             }
         }
     } else {   // ---------------- softmax warps 2..9: two threads per query row ----------------
@@ -234,9 +245,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
         // the two warps of a quarter meet on their own named barrier (ids 2..5)
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory"); };
         pdl_wait();
-        {   // Q -> shared memory, K-major with the 128-byte swizzle (16-byte chunk index XOR row % 8), value + residual.
-            // Both threads of a row read the whole head (the norm and the rotation need all of it) and each writes the
-            // eight 16-byte chunks of its own half.
+        {   // Q -> tensor memory, value + residual.  Both threads of a row read the whole head (the norm and the rotation
+            // need all of it) and each writes its own half.
             const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
             const float *src = p.qkv + ((size_t)seq * p.T + (size_t)min(tok, p.T - 1)) * p.row_stride + (size_t)h * kHeadDim;
             float q[128];
@@ -261,22 +271,24 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                     q[64 + i] = b0 * t.x + a0 * t.y; q[65 + i] = b1 * t.z + a1 * t.w;
                 }
             }
+            // this thread's 64 elements: value pairs to columns 32 * half .. + 31 of the first block, residual pairs to
+            // the same columns of the second
+            const uint32_t tqw = tmem_base + lane_addr + kColQ + 32u * half;
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-                float f[8];
+            for (int i = 0; i < 2; ++i) {
+                uint32_t qh[16], ql[16];
 #pragma unroll
-                for (int e = 0; e < 8; ++e)   // compile-time indices on both sides keep q[] in registers; half is warp-uniform
-                    f[e] = valid ? (half ? q[64 + 8 * cc + e] : q[8 * cc + e]) * qscale : 0.f;
-                uint4 hi, lo;
-                hi.x = pack_bf16x2(f[0], f[1]); lo.x = pack_bf16x2(f[0] - bf16_lo(hi.x), f[1] - bf16_hi(hi.x));
-                hi.y = pack_bf16x2(f[2], f[3]); lo.y = pack_bf16x2(f[2] - bf16_lo(hi.y), f[3] - bf16_hi(hi.y));
-                hi.z = pack_bf16x2(f[4], f[5]); lo.z = pack_bf16x2(f[4] - bf16_lo(hi.z), f[5] - bf16_hi(hi.z));
-                hi.w = pack_bf16x2(f[6], f[7]); lo.w = pack_bf16x2(f[6] - bf16_lo(hi.w), f[7] - bf16_hi(hi.w));
-                const uint32_t off = (uint32_t)half * kSlab + (uint32_t)r * 128u + (uint32_t)((cc ^ (r & 7)) << 4);
-                sts128(q_hi + off, hi);
-                sts128(q_lo + off, lo);
+                for (int e = 0; e < 16; ++e) {   // compile-time indices on both sides keep q[] in registers; half is warp-uniform
+                    const float a = valid ? (half ? q[64 + 32 * i + 2 * e] : q[32 * i + 2 * e]) * qscale : 0.f;
+                    const float b = valid ? (half ? q[64 + 32 * i + 2 * e + 1] : q[32 * i + 2 * e + 1]) * qscale : 0.f;
+                    qh[e] = pack_bf16x2(a, b);
+                    ql[e] = pack_bf16x2(a - bf16_lo(qh[e]), b - bf16_hi(qh[e]));
+                }
+                tmem_st16(tqw + 16u * i, qh);
+                tmem_st16(tqw + 64u + 16u * i, ql);
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes, async-proxy (MMA) reads
+            tmem_wait_st();
+            tc_fence_before();
             mbar_arrive(q_ready);
         }
         float m_used = -INFINITY, l = 0.f;   // l: this thread's share of the row sum
@@ -285,7 +297,11 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
         bool dead = false;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1, u = j >> 1;
+            const unsigned long long ts0 = NNC_TRACE_NOW();
+            (void)ts0;
             if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(s_full(s), (uint32_t)(u & 1), abort_flag, p.status, 27));
+            const unsigned long long ts1 = NNC_TRACE_NOW();
+            (void)ts1;
             const uint32_t ts = tmem_base + lane_addr + kColS + (uint32_t)s * kKN;
             float sv[64];
             float m_tile = -INFINITY;
@@ -353,9 +369,14 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 uint32_t ph[16], pl[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float a = sv[32 * i + 2 * e], b = sv[32 * i + 2 * e + 1];
-                    ph[e] = pack_bf16x2(a, b);
-                    pl[e] = pack_bf16x2(a - bf16_lo(ph[e]), b - bf16_hi(ph[e]));
+                    // value = the upper 16 bits of the fp32 pattern (truncation), residual = the upper 16 bits of
+                    // what is left: byte permutes and two subtractions, nothing on the conversion pipe, which the
+                    // exponentials keep busy.  value + residual still carries 15-16 bits of the probability.
+                    const uint32_t a = __float_as_uint(sv[32 * i + 2 * e]), b = __float_as_uint(sv[32 * i + 2 * e + 1]);
+                    ph[e] = __byte_perm(a, b, 0x7632);
+                    const float ra = __uint_as_float(a) - __uint_as_float(a & 0xffff0000u);
+                    const float rb = __uint_as_float(b) - __uint_as_float(b & 0xffff0000u);
+                    pl[e] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
                 }
                 tmem_st16(ts + 32u * half + 16u * i, ph);
                 tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
@@ -363,6 +384,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(p_full(s));
+            if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && warp == 2 && lane == 0) NNC_TRACE_EVENT(303, ts0, ts1, NNC_TRACE_NOW());
         }
         bool ok = !dead;
         // ---- O / l -> output: the pair adds its partial row sums, each thread writes its 64 columns ----
