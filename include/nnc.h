@@ -265,6 +265,12 @@ int nnc_op_attn_prefill(const float *qkv, const void *kcache, const void *vcache
                         int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_past,
                         void *cuda_stream);
 
+/* The one-term form the prompt phase uses: k16, v16 fp16 images of the cache rows (same layout; exact for bf16 values
+ * inside the fp16 range), queries and probabilities travel as one fp16 term each (half the tensor-core work of the form
+ * above), out fp16 [batch * T][n_q_heads * 128]. */
+int nnc_op_attn_prefill_f16(const float *qkv, const void *k16, const void *v16, void *out, int32_t batch, int32_t T,
+                            int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_past, void *cuda_stream);
+
 /* The same operation for callers that cannot allocate device memory (the paper has no counterpart: this is a
  * deployment convenience of this library).  A plug-in that is handed only its inputs and outputs, or a process
  * whose device memory is owned by another runtime's pool, cannot produce the scratch buffer above; here the

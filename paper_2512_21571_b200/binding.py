@@ -84,6 +84,8 @@ EXPORTS = {
                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "nnc_op_attn_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
+    "nnc_op_attn_prefill_f16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "nnc_op_attn_decode_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
 }
@@ -391,3 +393,12 @@ def op_attn_prefill(qkv: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tenso
                                 out.data_ptr(), out_lo.data_ptr(), batch, T, n_q_heads, nkv, max_seq, n_past,
                                 _stream_ptr()), "nnc_op_attn_prefill")
     return out, out_lo
+
+
+def op_attn_prefill_f16(qkv: torch.Tensor, k16: torch.Tensor, v16: torch.Tensor, T: int, n_q_heads: int, n_past: int):
+    """nnc_op_attn_prefill_f16; k16, v16 fp16 [batch][n_kv_heads][max_seq][128]; returns fp16 [batch * T][n_q_heads * 128]."""
+    batch, nkv, max_seq, _ = k16.shape
+    out = torch.empty(batch * T, n_q_heads * 128, dtype=torch.float16, device="cuda")
+    _ok(lib.nnc_op_attn_prefill_f16(_dev(qkv, torch.float32), _dev(k16, torch.float16), _dev(v16, torch.float16), out.data_ptr(),
+                                    batch, T, n_q_heads, nkv, max_seq, n_past, _stream_ptr()), "nnc_op_attn_prefill_f16")
+    return out

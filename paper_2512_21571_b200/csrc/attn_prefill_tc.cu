@@ -118,8 +118,10 @@ struct PfParams {
     int *status;
 };
 
-// OUT_FP16: the output is one fp16 matrix (saturating) instead of a bf16 value + residual pair
-template <bool OUT_FP16>
+// OUT_FP16: the output is one fp16 matrix (saturating) instead of a bf16 value + residual pair.
+// F16: the tensor maps cover an fp16 image of the K/V rows (exact for bf16 values inside the fp16 range), and Q and P
+// travel as ONE fp16 term each: half the tensor-core instructions of the two-bf16-term form.
+template <bool OUT_FP16, bool F16>
 __global__ void __launch_bounds__(kPfThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -185,8 +187,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc_qk = make_idesc(kKN, false, false);
-            constexpr uint32_t idesc_pv = make_idesc(kHeadDim, false, true);
+            constexpr uint32_t idesc_qk = make_idesc(kKN, F16, false);
+            constexpr uint32_t idesc_pv = make_idesc(kHeadDim, F16, true);
             bool ok = mbar_wait(q_ready, 0u, abort_flag, p.status, 22);
             tc_fence_after();
             // Descriptors differ only in their 14-bit start-address field (bytes >> 4), so every operand descriptor of
@@ -206,7 +208,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dimension elements per instruction
                     const uint64_t off = (uint64_t)(((ks >> 2) * kSlab + (ks & 3) * 32) >> 4);
                     umma_bf16_ts(d, tq + (uint32_t)ks * 8u, b0 + off, idesc_qk, ks != 0);
-                    umma_bf16_ts(d, tq + 64u + (uint32_t)ks * 8u, b0 + off, idesc_qk, 1u);
+                    if (!F16) umma_bf16_ts(d, tq + 64u + (uint32_t)ks * 8u, b0 + off, idesc_qk, 1u);
                 }
                 umma_commit(s_full(s));
                 return true;
@@ -228,7 +230,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int ks = 0; ks < 8; ++ks) {   // 16 cache positions per instruction
                     const uint64_t b = dv[s] + (uint64_t)(ks * (2048 >> 4));
                     umma_bf16_ts(d, pa + (uint32_t)ks * 8u, b, idesc_pv, (j != 0) || (ks != 0));
-                    umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
+                    if (!F16) umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
                 }
                 umma_commit(pv_done(s));
                 if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) NNC_TRACE_EVENT(302, tr0, tr1, NNC_TRACE_NOW());
@@ -281,11 +283,16 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int e = 0; e < 16; ++e) {   // compile-time indices on both sides keep q[] in registers; half is warp-uniform
                     const float a = valid ? (half ? q[64 + 32 * i + 2 * e] : q[32 * i + 2 * e]) * qscale : 0.f;
                     const float b = valid ? (half ? q[64 + 32 * i + 2 * e + 1] : q[32 * i + 2 * e + 1]) * qscale : 0.f;
-                    qh[e] = pack_bf16x2(a, b);
-                    ql[e] = pack_bf16x2(a - bf16_lo(qh[e]), b - bf16_hi(qh[e]));
+                    if (F16) {
+                        qh[e] = pack_f16x2_sat(a, b);
+                        ql[e] = 0u;
+                    } else {
+                        qh[e] = pack_bf16x2(a, b);
+                        ql[e] = pack_bf16x2(a - bf16_lo(qh[e]), b - bf16_hi(qh[e]));
+                    }
                 }
                 tmem_st16(tqw + 16u * i, qh);
-                tmem_st16(tqw + 64u + 16u * i, ql);
+                if (!F16) tmem_st16(tqw + 64u + 16u * i, ql);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -369,17 +376,22 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 uint32_t ph[16], pl[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    // value = the upper 16 bits of the fp32 pattern (truncation), residual = the upper 16 bits of
-                    // what is left: byte permutes and two subtractions, nothing on the conversion pipe, which the
-                    // exponentials keep busy.  value + residual still carries 15-16 bits of the probability.
-                    const uint32_t a = __float_as_uint(sv[32 * i + 2 * e]), b = __float_as_uint(sv[32 * i + 2 * e + 1]);
-                    ph[e] = __byte_perm(a, b, 0x7632);
-                    const float ra = __uint_as_float(a) - __uint_as_float(a & 0xffff0000u);
-                    const float rb = __uint_as_float(b) - __uint_as_float(b & 0xffff0000u);
-                    pl[e] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+                    if (F16) {   // probabilities are at most 2^8: inside the fp16 range
+                        ph[e] = pack_f16x2_sat(sv[32 * i + 2 * e], sv[32 * i + 2 * e + 1]);
+                        pl[e] = 0u;
+                    } else {
+                        // value = the upper 16 bits of the fp32 pattern (truncation), residual = the upper 16 bits of
+                        // what is left: byte permutes and two subtractions, nothing on the conversion pipe, which the
+                        // exponentials keep busy.  value + residual still carries 15-16 bits of the probability.
+                        const uint32_t a = __float_as_uint(sv[32 * i + 2 * e]), b = __float_as_uint(sv[32 * i + 2 * e + 1]);
+                        ph[e] = __byte_perm(a, b, 0x7632);
+                        const float ra = __uint_as_float(a) - __uint_as_float(a & 0xffff0000u);
+                        const float rb = __uint_as_float(b) - __uint_as_float(b & 0xffff0000u);
+                        pl[e] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+                    }
                 }
                 tmem_st16(ts + 32u * half + 16u * i, ph);
-                tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
+                if (!F16) tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -447,21 +459,21 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
 
 // bf16 cache of one layer as a 3-D tensor [heads = batch * nkv][positions][128]; only the first n_valid positions of
 // every head are inside the tensor, so the rest of a box arrives as zeros
-bool make_cache_map(CUtensorMap *map, const bf16 *cache, int heads, int n_valid, int max_seq) {
+bool make_cache_map(CUtensorMap *map, const void *cache, int heads, int n_valid, int max_seq, bool fp16) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_valid, (cuuint64_t)heads};
     const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)max_seq * kHeadDim * 2};
     const cuuint32_t box[3] = {64, (cuuint32_t)kKN, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16 *>(cache), dims, strides, box, estr,
+    return enc(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(cache), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool OUT_FP16>
+template <bool OUT_FP16, bool F16>
 cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensorMap &mv, const PfParams &p, dim3 grid) {
-    auto kern = attn_prefill_tc_kernel<OUT_FP16>;
+    auto kern = attn_prefill_tc_kernel<OUT_FP16, F16>;
     static unsigned long long attr_done = 0;   // per instantiation, one bit per device
     if (cudaError_t e = ensure_dynamic_smem(kern, kPfSmem, &attr_done); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -482,21 +494,24 @@ cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensor
 
 // rows = batch * rows_per_seq new tokens, the token of row s * rows_per_seq + i sitting at position n_past + i of
 // sequence s; the cache must already hold their K/V.  n_past is a host value: it sizes the tensor maps.
-cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
-                                const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
-                                int n_past, const AttnFused *fused) {
+// kv_f16: kcache / vcache point at an fp16 image of the cache rows (same layout) and the kernel runs its one-term form.
+cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const void *kcache,
+                                const void *vcache, bool kv_f16, void *out, void *out_lo, bool out_fp16, int nq, int nkv,
+                                int max_seq, int n_past, const AttnFused *fused) {
     const int batch = rows / rows_per_seq, T = rows_per_seq;
     if (T <= 0 || batch <= 0 || n_past < 0 || n_past + T > max_seq || nq % nkv) return cudaErrorInvalidValue;
     if (((uintptr_t)qkv | (uintptr_t)kcache | (uintptr_t)vcache | (uintptr_t)out | (uintptr_t)out_lo) & 15) return cudaErrorInvalidValue;
     CUtensorMap mk, mv;
-    if (!make_cache_map(&mk, kcache, batch * nkv, n_past + T, max_seq) || !make_cache_map(&mv, vcache, batch * nkv, n_past + T, max_seq))
+    if (!make_cache_map(&mk, kcache, batch * nkv, n_past + T, max_seq, kv_f16) ||
+        !make_cache_map(&mv, vcache, batch * nkv, n_past + T, max_seq, kv_f16))
         return cudaErrorInvalidValue;
     PfParams p;
     p.qkv = qkv; p.row_stride = (nq + 2 * nkv) * kHeadDim; p.out = out; p.out_lo = out_lo;
     p.T = T; p.n_past = n_past; p.nq = nq; p.nkv = nkv; p.status = lc.status;
     p.g_q = fused ? fused->g_q : nullptr; p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;
     const dim3 grid((T + kQM - 1) / kQM, nq, batch);
-    return out_fp16 ? launch_pf<true>(lc, mk, mv, p, grid) : launch_pf<false>(lc, mk, mv, p, grid);
+    if (kv_f16) return out_fp16 ? launch_pf<true, true>(lc, mk, mv, p, grid) : launch_pf<false, true>(lc, mk, mv, p, grid);
+    return out_fp16 ? launch_pf<true, false>(lc, mk, mv, p, grid) : launch_pf<false, false>(lc, mk, mv, p, grid);
 }
 
 }  // namespace nnc

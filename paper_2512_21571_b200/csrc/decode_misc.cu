@@ -37,7 +37,8 @@ __global__ void __launch_bounds__(128)
 qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, const bf16 *__restrict__ g_q,
                            const bf16 *__restrict__ g_k, float eps, const float *__restrict__ rope,
                            bf16 *__restrict__ kcache, bf16 *__restrict__ vcache, int nq, int nkv, int max_seq,
-                           const int32_t *__restrict__ d_len, int skip_q) {
+                           const int32_t *__restrict__ d_len, int skip_q, uint16_t *__restrict__ k16,
+                           uint16_t *__restrict__ v16) {
     NNC_TRACE_SCOPE(2);
     pdl_wait();
     const int heads = nq + 2 * nkv;
@@ -72,9 +73,16 @@ qk_norm_rope_append_kernel(float *__restrict__ qkv, int rows, int rows_per_seq, 
             } else {
                 const bool is_k = head < nq + nkv;
                 const int j = is_k ? head - nq : head - nq - nkv;
-                bf16 *dst = (is_k ? kcache : vcache) + (((size_t)seq * nkv + j) * max_seq + pos) * kHeadDim;
-                reinterpret_cast<uint32_t *>(dst)[lane] = pack_bf16x2(a.x, a.y);
-                reinterpret_cast<uint32_t *>(dst + 64)[lane] = pack_bf16x2(b.x, b.y);
+                const size_t off = (((size_t)seq * nkv + j) * max_seq + pos) * kHeadDim;
+                bf16 *dst = (is_k ? kcache : vcache) + off;
+                const uint32_t pa = pack_bf16x2(a.x, a.y), pb = pack_bf16x2(b.x, b.y);
+                reinterpret_cast<uint32_t *>(dst)[lane] = pa;
+                reinterpret_cast<uint32_t *>(dst + 64)[lane] = pb;
+                uint16_t *d16 = is_k ? k16 : v16;
+                if (d16) {   // fp16 image of the bf16 row just written (the same values wherever fp16 can hold them)
+                    reinterpret_cast<uint32_t *>(d16 + off)[lane] = pack_f16x2_sat(bf16_lo(pa), bf16_hi(pa));
+                    reinterpret_cast<uint32_t *>(d16 + off + 64)[lane] = pack_f16x2_sat(bf16_lo(pb), bf16_hi(pb));
+                }
             }
         }
     }
@@ -146,6 +154,20 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
     for (int i = threadIdx.x + 256 * kKeep; i < n4; i += 256) emit(i, src[i]);
 }
 
+// dst[h][pos][:] = fp16(src[h][pos][:]) for pos < n_pos; 16 bytes (8 elements) per thread
+__global__ void kv_rows_to_f16_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int heads, int max_seq, int n_pos) {
+    pdl_wait();
+    const size_t per_head = (size_t)n_pos * (kHeadDim / 8), total = per_head * heads;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t h = i / per_head, r = i % per_head;
+        const size_t at = h * (size_t)max_seq * (kHeadDim / 8) + r;
+        const uint4 v = src[at];
+        dst[at] = make_uint4(pack_f16x2_sat(bf16_lo(v.x), bf16_hi(v.x)), pack_f16x2_sat(bf16_lo(v.y), bf16_hi(v.y)),
+                             pack_f16x2_sat(bf16_lo(v.z), bf16_hi(v.z)), pack_f16x2_sat(bf16_lo(v.w), bf16_hi(v.w)));
+    }
+    pdl_launch_dependents();
+}
+
 __global__ void copy_f32_kernel(const float *__restrict__ src, float *__restrict__ dst, size_t n) {
     pdl_wait();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
@@ -169,16 +191,25 @@ cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *toke
 cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
-                                       const int32_t *d_len, bool skip_q) {
+                                       const int32_t *d_len, bool skip_q, void *k16, void *v16) {
     const long units = (long)rows * (skip_q ? 2 * nkv : nq + 2 * nkv);
     return launch(lc, qk_norm_rope_append_kernel, dim3((unsigned)((units + 3) / 4)), dim3(128), qkv, rows,
-                  rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, skip_q ? 1 : 0);
+                  rows_per_seq, g_q, g_k, eps, rope, kcache_layer, vcache_layer, nq, nkv, max_seq, d_len, skip_q ? 1 : 0,
+                  (uint16_t *)k16, (uint16_t *)v16);
 }
 
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
                                 int H, float eps, int first, int step, bool out_f16) {
     if (out_f16) return launch(lc, rmsnorm_rows_kernel<true>, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
     return launch(lc, rmsnorm_rows_kernel<false>, dim3(rows), dim3(256), x, gain, out, out_lo, H, eps, first, step);
+}
+
+cudaError_t launch_kv_rows_to_f16(const LaunchCtx &lc, const bf16 *src, void *dst, int heads, int max_seq, int n_pos) {
+    if (n_pos <= 0) return cudaSuccess;
+    size_t blocks = ((size_t)heads * n_pos * (kHeadDim / 8) + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    return launch(lc, kv_rows_to_f16_kernel, dim3((unsigned)blocks), dim3(256), reinterpret_cast<const uint4 *>(src),
+                  reinterpret_cast<uint4 *>(dst), heads, max_seq, n_pos);
 }
 
 cudaError_t launch_copy_f32(const LaunchCtx &lc, const float *src, float *dst, size_t n) {

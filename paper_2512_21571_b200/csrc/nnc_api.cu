@@ -39,7 +39,7 @@ struct Plan {
     // offsets
     std::vector<size_t> l_wqkv, l_wo, l_wgu, l_wd, l_gin, l_gpost, l_gq, l_gk, l_wo16, l_wgu16, l_wd16;
     std::vector<size_t> l_q8, l_s8;   // FP8: codes of the four matrices back to back, then their row scales
-    size_t f16_scales, f16_word, lm_q8, lm_s8;
+    size_t f16_scales, f16_word, lm_q8, lm_s8, k16, v16;
     size_t embed, lm_head, g_final, kcache, vcache, rope;
     size_t gemv_ctr, gemm_part, gemm_tickets, x, qkv, attn_out, act, part, tickets, am_val, am_idx, am_ticket, d_len, d_status, d_tokens, d_argmax;
     size_t xt, hb, hb_lo, qkvt, ob, ob_lo, ab, ab_lo, logits_stage;
@@ -94,6 +94,9 @@ void make_plan(const nnc_config &c, Plan &p) {
     }
     p.lm_q8 = p.take(c.weight_format == 1 ? V * H : 0);
     p.lm_s8 = p.take(c.weight_format == 1 ? V * sizeof(float) : 0);
+    // fp16 image of ONE layer's K/V rows, rebuilt per layer by the prompt phase (its attention runs in fp16)
+    p.k16 = p.take(wants_f16_copies(c) ? B * kd * c.max_seq * 2 : 0);
+    p.v16 = p.take(wants_f16_copies(c) ? B * kd * c.max_seq * 2 : 0);
     p.f16_scales = p.take((size_t)c.n_layers * 3 * 2 * sizeof(float));
     p.f16_word = p.take(4);
     p.embed = p.take(V * H * 2);
@@ -151,6 +154,7 @@ struct nnc_model {
     bf16 *hb, *ob, *ab;
     bf16 *hb_lo, *ob_lo, *ab_lo;  // bf16 rounding residuals of the GEMM activations (null in the one-term mode)
     bool f16_copies;              // the layers hold fp16 copies of Wo, Wgate/up, Wdown
+    void *k16, *v16;              // fp16 image of one layer's K/V rows (prompt phase with fp16 operands; null otherwise)
     uint8_t *lm_q8;               // weight_format 1: FP8 codes and row scales of the lm_head (null otherwise)
     float *lm_s8;
     int len;
@@ -248,10 +252,17 @@ int forward_tokens(nnc_model *m, const int32_t *tokens, int batch, int T, float 
                                            batch, c.n_q_heads, c.n_kv_heads, c.max_seq, n_splits, &fused));
         } else {
             // K/V heads: norm, rotation, append; the query heads are normalised and rotated by the attention kernel
+            // With fp16 operands the attention reads an fp16 image of this layer's K/V rows: the new rows are written
+            // there by the append kernel, rows of earlier calls are converted first.
+            if (f16 && m->len > 0) {
+                NNC_CUDA(m, launch_kv_rows_to_f16(lc, kc, m->k16, batch * c.n_kv_heads, c.max_seq, m->len));
+                NNC_CUDA(m, launch_kv_rows_to_f16(lc, vc, m->v16, batch * c.n_kv_heads, c.max_seq, m->len));
+            }
             NNC_CUDA(m, launch_qk_norm_rope_append(lc, m->qkvt, R, T, w.g_q, w.g_k, c.rms_eps, m->rope, kc, vc, c.n_q_heads,
-                                                   c.n_kv_heads, c.max_seq, m->d_len, true));
+                                                   c.n_kv_heads, c.max_seq, m->d_len, true, f16 ? m->k16 : nullptr, f16 ? m->v16 : nullptr));
             const AttnFused fused{w.g_q, w.g_k, m->rope, c.rms_eps};
-            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, kc, vc, m->ob, f16 ? nullptr : m->ob_lo, f16, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len, &fused));
+            NNC_CUDA(m, launch_attn_prefill(lc, m->qkvt, R, T, f16 ? (const void *)m->k16 : kc, f16 ? (const void *)m->v16 : vc, f16, m->ob,
+                                            f16 ? nullptr : m->ob_lo, f16, c.n_q_heads, c.n_kv_heads, c.max_seq, m->len, &fused));
         }
         if (f16) {
             NNC_CUDA(m, launch_gemm(lc, m->ob, nullptr, (const bf16 *)w.wo16, m->xt, nullptr, R, H, qd, H, kEpiAccumF32, m->d_status, nullptr, true, w.sc_o + 1));
@@ -355,6 +366,8 @@ int nnc_model_create(const nnc_config *config, const nnc_weights *weights, void 
                 w.s_qkv = (float *)at(p.l_s8[l]); w.s_o = w.s_qkv + qkvd; w.s_gu = w.s_o + Hs; w.s_d = w.s_gu + 2 * Is;
             }
         }
+        m->k16 = wants_f16_copies(c) ? at(p.k16) : nullptr;
+        m->v16 = wants_f16_copies(c) ? at(p.v16) : nullptr;
         m->lm_q8 = c.weight_format == 1 ? (uint8_t *)at(p.lm_q8) : nullptr;
         m->lm_s8 = c.weight_format == 1 ? (float *)at(p.lm_s8) : nullptr;
         m->embed = (bf16 *)at(p.embed); m->lm_head = (bf16 *)at(p.lm_head); m->g_final = (bf16 *)at(p.g_final);
@@ -836,6 +849,18 @@ int nnc_op_gemv(const void *W, const float *x, float *y, int32_t n_out, int32_t 
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }
 
+int nnc_op_attn_prefill_f16(const float *qkv, const void *k16, const void *v16, void *out, int32_t batch, int32_t T,
+                            int32_t n_q_heads, int32_t n_kv_heads, int32_t max_seq, int32_t n_past, void *cuda_stream) {
+    if (!qkv || !k16 || !v16 || !out) return NNC_ERR_INVALID_ARG;
+    if (batch <= 0 || T <= 0 || n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % n_kv_heads || n_past < 0) return NNC_ERR_INVALID_ARG;
+    if ((long)n_past + T > max_seq) return NNC_ERR_CAPACITY;
+    LaunchCtx lc;
+    if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
+    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, k16, v16, true, out, nullptr, true, n_q_heads, n_kv_heads, max_seq, n_past);
+    if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
+    return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
+}
+
 int nnc_op_gemv_fp8(const void *codes, const float *scales, const float *x, float *y, int32_t n_out, int32_t n_in,
                     const void *gain, float eps, int32_t mode, void *cuda_stream) {
     const bool chained = (mode & NNC_GEMV_CHAINED) != 0;
@@ -893,8 +918,8 @@ int nnc_op_attn_prefill(const float *qkv, const void *kcache, const void *vcache
     if ((long)n_past + T > max_seq) return NNC_ERR_CAPACITY;
     LaunchCtx lc;
     if (op_ctx(lc, cuda_stream)) return NNC_ERR_CUDA;
-    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, (const bf16 *)kcache, (const bf16 *)vcache, out, out_lo, false,
-                                        n_q_heads, n_kv_heads, max_seq, n_past);
+    cudaError_t e = launch_attn_prefill(lc, qkv, batch * T, T, kcache, vcache, false, out, out_lo, false, n_q_heads, n_kv_heads,
+                                        max_seq, n_past);
     if (e == cudaErrorInvalidValue) return NNC_ERR_INVALID_ARG;
     return e == cudaSuccess ? NNC_OK : NNC_ERR_CUDA;
 }

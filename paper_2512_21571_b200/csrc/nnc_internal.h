@@ -82,10 +82,11 @@ cudaError_t launch_quantise_rows_e4m3(const LaunchCtx &lc, const bf16 *W, uint8_
 cudaError_t launch_embed(const LaunchCtx &lc, const bf16 *E, const int32_t *tokens, float *x, int rows, int H,
                          int vocab, float *tap);
 // skip_q: only the key and value heads are processed (the consumer of the queries normalises and rotates them itself)
+// k16 / v16 (nullable): fp16 images of one layer's cache (same layout); the appended rows are written there as well
 cudaError_t launch_qk_norm_rope_append(const LaunchCtx &lc, float *qkv, int rows, int rows_per_seq,
                                        const bf16 *g_q, const bf16 *g_k, float eps, const float *rope,
                                        bf16 *kcache_layer, bf16 *vcache_layer, int nq, int nkv, int max_seq,
-                                       const int32_t *d_len, bool skip_q);
+                                       const int32_t *d_len, bool skip_q, void *k16 = nullptr, void *v16 = nullptr);
 // out_f16: `out` receives one fp16 matrix (saturating) instead of a bf16 value (+ residual in out_lo)
 cudaError_t launch_rmsnorm_rows(const LaunchCtx &lc, const float *x, const bf16 *gain, bf16 *out, bf16 *out_lo, int rows,
                                 int H, float eps, int first, int step, bool out_f16 = false);
@@ -112,9 +113,13 @@ cudaError_t launch_attn_decode(const LaunchCtx &lc, const float *q, int q_row_st
 // or, with out_fp16, one fp16 matrix.  n_past (cached positions before this call) is a host value: it sizes the tensor maps.
 // fused != null: the query heads of qkv are raw projections and the kernel applies the per-head RMSNorm (g_q) and RoPE
 // itself (the K/V rows must already be in the cache: launch_qk_norm_rope_append with skip_q).
-cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const bf16 *kcache,
-                                const bf16 *vcache, void *out, void *out_lo, bool out_fp16, int nq, int nkv, int max_seq,
-                                int n_past, const AttnFused *fused = nullptr);
+// kv_f16: kcache / vcache point at an fp16 image of the cache rows (same [batch][nkv][max_seq][128] layout) and Q and P
+// travel as one fp16 term each; otherwise they are the bf16 cache and Q and P travel as two bf16 terms.
+cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows, int rows_per_seq, const void *kcache,
+                                const void *vcache, bool kv_f16, void *out, void *out_lo, bool out_fp16, int nq, int nkv,
+                                int max_seq, int n_past, const AttnFused *fused = nullptr);
+// fp16 image of cache rows [0, n_pos) of every (sequence, KV head): dst and src share the [heads][max_seq][128] layout
+cudaError_t launch_kv_rows_to_f16(const LaunchCtx &lc, const bf16 *src, void *dst, int heads, int max_seq, int n_pos);
 
 // ---- GEMM (gemm_tc.cu) --------------------------------------------------------------------------------
 enum GemmEpi { kEpiStoreF32 = 0, kEpiStoreBf16 = 1, kEpiAccumF32 = 2, kEpiSwigluBf16 = 3 };

@@ -51,10 +51,11 @@ def test_workspace_bytes_is_host_arithmetic(binding):
     assert n2 - n >= kv
     tied = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, tie_embeddings=1)))
     assert n - tied == 151936 * 4096 * 2
-    # prompt-phase capacity beyond 128 tokens adds the fp16 copies of Wo, Wgate/up, Wdown in operand mode 0 only
+    # prompt-phase capacity beyond 128 tokens adds, in operand mode 0 only, the fp16 copies of Wo, Wgate/up, Wdown and
+    # the fp16 image of one layer's K and V rows
     big0 = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, max_tokens=8192)))
     big1 = binding.lib.nnc_workspace_bytes(C.byref(_cfg(binding, max_tokens=8192, tc_operands=1)))
-    assert big0 - big1 == 2 * 36 * (4096 * 4096 + 3 * 12288 * 4096)
+    assert big0 - big1 == 2 * 36 * (4096 * 4096 + 3 * 12288 * 4096) + 2 * (8 * 128 * 4352 * 2)
 
 
 @pytest.mark.parametrize("bad", [dict(head_dim=64), dict(n_q_heads=30), dict(hidden=1000), dict(max_seq=0),
