@@ -469,31 +469,39 @@ def kernel_roofline_attn(shape, peaks, batch, ctx):
 
 
 def kernel_roofline_attn_prefill(shape, peaks, batch, T):
-    """The prompt-phase attention kernel timed alone: causal attention of `batch` sequences of T new tokens (no past).
-    Model FLOPs = 4 * 128 * T (T + 1) / 2 per head; the kernel issues twice that (Q and P travel as two bf16 terms)."""
+    """The prompt-phase attention kernel timed alone: causal attention of `batch` sequences of T new tokens (no past),
+    in the one-fp16-term form the prompt phase uses and, beside it, the two-bf16-term form.  Model FLOPs =
+    4 * 128 * T (T + 1) / 2 per head."""
     from paper_2512_21571_b200 import binding
     nq, nkv = shape.n_q_heads, shape.n_kv_heads
     qkv = synth.normal(9, 21, (batch * T, (nq + 2 * nkv) * 128), 1.0, torch.float32, "cuda")
     kc = synth.normal(9, 22, (batch, nkv, T, 128), 1.0, torch.bfloat16, "cuda")
     vc = synth.normal(9, 23, (batch, nkv, T, 128), 1.0, torch.bfloat16, "cuda")
-    for _ in range(3):
-        binding.op_attn_prefill(qkv, kc, vc, T, nq, 0)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k16, v16 = kc.to(torch.float16), vc.to(torch.float16)
+    runs = {"f16": lambda: binding.op_attn_prefill_f16(qkv, k16, v16, T, nq, 0),
+            "bf16_two_terms": lambda: binding.op_attn_prefill(qkv, kc, vc, T, nq, 0)}
+    us = {}
     n = 10
-    e0.record()
-    for _ in range(n):
-        binding.op_attn_prefill(qkv, kc, vc, T, nq, 0)
-    e1.record()
-    torch.cuda.synchronize()
+    for name, fn in runs.items():
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        us[name] = e0.elapsed_time(e1) * 1e3 / n
     assert binding.op_status() == 0
-    us = e0.elapsed_time(e1) * 1e3 / n
     flops = 4.0 * 128 * batch * nq * (T * (T + 1) / 2)
-    ach = flops / (us * 1e-6) / 1e12
-    return {"bound": "tensor", "kernel": "attn_prefill_tc_kernel", "shape": [batch, nq, T, 128], "achieved": round(ach, 1),
-            "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ach / peaks["bf16_tflops"], 4),
-            "peak_source": peaks["source"] + " (burst)", "flops_per_launch": flops, "issued_tflops": round(2 * ach, 1),
-            "us_per_launch": round(us, 1), "launches_timed": n,
+    ach = flops / (us["f16"] * 1e-6) / 1e12
+    return {"bound": "tensor", "kernel": "attn_prefill_tc_kernel<one fp16 term>", "shape": [batch, nq, T, 128],
+            "achieved": round(ach, 1), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ach / peaks["bf16_tflops"], 4),
+            "peak_source": peaks["source"] + " (burst)", "flops_per_launch": flops,
+            "us_per_launch": round(us["f16"], 1), "launches_timed": n,
+            "bf16_two_terms": {"us_per_launch": round(us["bf16_two_terms"], 1),
+                               "model_tflops": round(flops / (us["bf16_two_terms"] * 1e-6) / 1e12, 1)},
             "traffic": measured_traffic("attn_prefill_tc_kernel:b%d_T%d" % (batch, T))}
 
 
