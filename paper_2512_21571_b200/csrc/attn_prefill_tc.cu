@@ -28,95 +28,18 @@
 // tile's maximum exceeds it by more than 2^8; probabilities then stay below 256, which fp32 sums and the bf16
 // pair hold without loss.  The result is the exact softmax whatever m is.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains and frees its tensor memory.
-#include "tc_common.cuh"
+#include "attn_prefill_common.cuh"
 
 namespace nnc {
 
 namespace {
 
-constexpr int kQM = 128;                 // query rows per CTA
-constexpr int kKN = 128;                 // cache positions per tile
 constexpr int kPfThreads = 320;
 constexpr int kSoftmaxThreads = 256;
-constexpr int kSlab = 128 * 128;         // bytes of a [128 rows][64 x 16 bit] swizzled slab
-constexpr int kTile = 2 * kSlab;         // [128][128] 16-bit tile = two slabs (head-dimension halves)
 constexpr int kPfSmem = 4 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   // 2 x (K, V)
 // tensor-memory columns: two score / probability buffers, the output accumulator, the queries (value pairs in the
 // first 64 columns, residual pairs in the next 64; two head-dimension elements per column)
 constexpr uint32_t kColS = 0, kColO = 256, kColQ = 384, kTmemCols = 512;
-constexpr float kLazyMax = 8.f;          // log2 units
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
-        : "memory");
-}
-
-// tcgen05.mma with the A operand in tensor memory (K-major, two 16-bit elements per 32-bit column)
-__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// Shared-memory descriptor of an MN-major 16-bit operand under the 128-byte swizzle: 64 elements (128 bytes) are
-// contiguous along MN, the next 64 follow `lbo` bytes later; along K, rows are 128 bytes apart and groups of 8 rows
-// 1024 bytes.  That is exactly a [position][64] TMA box of cache rows, with the head-dimension halves one slab apart.
-__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr, uint32_t lbo) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-// tensor-memory load of 32 columns WITHOUT the wait: several may be issued back to back before one tmem_wait_ld()
-__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-struct PfParams {
-    const float *qkv;   // [batch * T][row_stride]: query heads first
-    int row_stride;     // floats per token row = (nq + 2 nkv) * 128
-    void *out, *out_lo; // [batch * T][nq * 128]: bf16 value (+ residual, nullable), or fp16
-    int T, n_past, nq, nkv;
-    const bf16 *g_q;    // not null: the queries are raw projections; apply RMSNorm (this gain) and RoPE while loading
-    const float *rope;  // [max_seq][64][2] (cos, sin), read when g_q is set
-    float eps;
-    int *status;
-};
 
 // OUT_FP16: the output is one fp16 matrix (saturating) instead of a bf16 value + residual pair.
 // F16: the tensor maps cover an fp16 image of the K/V rows (exact for bf16 values inside the fp16 range), and Q and P
@@ -141,8 +64,12 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
-    const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;   // longest rows first
-    const int h = blockIdx.y, seq = blockIdx.z;
+    // The grid is one-dimensional and ordered by decreasing length: all (head, sequence) pairs of the last query tile
+    // (the most cache tiles) first, the first query tile last, so that the long CTAs never start late.  Neighbouring
+    // CTAs are query heads of the same KV head: they stream the same cache tiles at the same time.
+    const int per_qt = p.nq * p.batch;
+    const int qt = p.n_qt - 1 - (int)blockIdx.x / per_qt;
+    const int h = ((int)blockIdx.x % per_qt) % p.nq, seq = ((int)blockIdx.x % per_qt) / p.nq;
     const int G = p.nq / p.nkv, jkv = h / G;
     const int q0 = qt * kQM;
     const int n_valid = p.n_past + p.T;
@@ -233,7 +160,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                     if (!F16) umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
                 }
                 umma_commit(pv_done(s));
-                if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) NNC_TRACE_EVENT(302, tr0, tr1, NNC_TRACE_NOW());
+                if (blockIdx.x == 0) NNC_TRACE_EVENT(302, tr0, tr1, NNC_TRACE_NOW());
             }
         }
     } else {   // ---------------- softmax warps 2..9: two threads per query row ----------------
@@ -326,8 +253,14 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                     for (int e = 0; e < 64; ++e)
                         if (k0 + e > pos) sv[e] = -INFINITY;
                 }
+                // four independent chains: with two softmax warps per scheduler a 64-long dependent chain is not hidden
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int e = 0; e < 64; ++e) m_tile = fmaxf(m_tile, sv[e]);
+                for (int e = 0; e < 64; e += 4) {
+                    mx[0] = fmaxf(mx[0], sv[e]); mx[1] = fmaxf(mx[1], sv[e + 1]);
+                    mx[2] = fmaxf(mx[2], sv[e + 2]); mx[3] = fmaxf(mx[3], sv[e + 3]);
+                }
+                m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 xch[s][half][r] = m_tile;
             }
             // After this barrier both threads of a row hold their scores in registers, so the probability columns may
@@ -365,10 +298,14 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                     m_used = m_new;
                 }
             }
-            float sum = 0.f;
+            // exponents are <= 2^8 by the lazy maximum; results below 2^-126 flush to zero, which a row sum >= 1 cannot see
+            float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int e = 0; e < 64; ++e) { sv[e] = exp2f(sv[e] - m_used); sum += sv[e]; }
-            l += sum;
+            for (int e = 0; e < 64; e += 4) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { sv[e + c] = ex2_approx(sv[e + c] - m_used); sum[c] += sv[e + c]; }
+            }
+            l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             // P over S: value pairs in columns 0..63, residual pairs in columns 64..127 (two positions per column);
             // this thread's 64 positions are columns 32 * half .. + 31 of each
 #pragma unroll
@@ -396,7 +333,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(p_full(s));
-            if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && warp == 2 && lane == 0) NNC_TRACE_EVENT(303, ts0, ts1, NNC_TRACE_NOW());
+            if (blockIdx.x == 0 && warp == 2 && lane == 0) NNC_TRACE_EVENT(303, ts0, ts1, NNC_TRACE_NOW());
         }
         bool ok = !dead;
         // ---- O / l -> output: the pair adds its partial row sums, each thread writes its 64 columns ----
@@ -457,20 +394,6 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
     }
 }
 
-// bf16 cache of one layer as a 3-D tensor [heads = batch * nkv][positions][128]; only the first n_valid positions of
-// every head are inside the tensor, so the rest of a box arrives as zeros
-bool make_cache_map(CUtensorMap *map, const void *cache, int heads, int n_valid, int max_seq, bool fp16) {
-    EncodeTiledFn enc = get_encode();
-    if (!enc) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_valid, (cuuint64_t)heads};
-    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)max_seq * kHeadDim * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kKN, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(cache), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <bool OUT_FP16, bool F16>
 cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensorMap &mv, const PfParams &p, dim3 grid) {
     auto kern = attn_prefill_tc_kernel<OUT_FP16, F16>;
@@ -509,8 +432,9 @@ cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows,
     p.qkv = qkv; p.row_stride = (nq + 2 * nkv) * kHeadDim; p.out = out; p.out_lo = out_lo;
     p.T = T; p.n_past = n_past; p.nq = nq; p.nkv = nkv; p.status = lc.status;
     p.g_q = fused ? fused->g_q : nullptr; p.rope = fused ? fused->rope : nullptr; p.eps = fused ? fused->eps : 0.f;
-    const dim3 grid((T + kQM - 1) / kQM, nq, batch);
-    if (kv_f16) return out_fp16 ? launch_pf<true, true>(lc, mk, mv, p, grid) : launch_pf<false, true>(lc, mk, mv, p, grid);
+    p.batch = batch; p.n_qt = (T + kQM - 1) / kQM;
+    const dim3 grid((unsigned)(p.n_qt * nq * batch));
+    if (kv_f16) return launch_attn_prefill_f16(lc, mk, mv, p, grid, out_fp16);
     return out_fp16 ? launch_pf<true, false>(lc, mk, mv, p, grid) : launch_pf<false, false>(lc, mk, mv, p, grid);
 }
 
