@@ -496,13 +496,13 @@ def kernel_roofline_attn_prefill(shape, peaks, batch, T):
     assert binding.op_status() == 0
     flops = 4.0 * 128 * batch * nq * (T * (T + 1) / 2)
     ach = flops / (us["f16"] * 1e-6) / 1e12
-    return {"bound": "tensor", "kernel": "attn_prefill_tc_kernel<one fp16 term>", "shape": [batch, nq, T, 128],
+    return {"bound": "tensor", "kernel": "attn_prefill_f16_kernel (one fp16 term; beside it attn_prefill_tc_kernel, two bf16 terms)", "shape": [batch, nq, T, 128],
             "achieved": round(ach, 1), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ach / peaks["bf16_tflops"], 4),
             "peak_source": peaks["source"] + " (burst)", "flops_per_launch": flops,
             "us_per_launch": round(us["f16"], 1), "launches_timed": n,
             "bf16_two_terms": {"us_per_launch": round(us["bf16_two_terms"], 1),
                                "model_tflops": round(flops / (us["bf16_two_terms"] * 1e-6) / 1e12, 1)},
-            "traffic": measured_traffic("attn_prefill_tc_kernel:b%d_T%d" % (batch, T))}
+            "traffic": measured_traffic("attn_prefill_f16_kernel:b%d_T%d" % (batch, T))}
 
 
 # ---- the CPU oracle leg (reported baseline; the only place the product's bench touches oracle/) ------------

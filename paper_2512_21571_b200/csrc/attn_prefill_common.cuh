@@ -91,12 +91,12 @@ struct PfParams {
 
 // bf16 cache of one layer as a 3-D tensor [heads = batch * nkv][positions][128]; only the first n_valid positions of
 // every head are inside the tensor, so the rest of a box arrives as zeros
-inline bool make_cache_map(CUtensorMap *map, const void *cache, int heads, int n_valid, int max_seq, bool fp16) {
+inline bool make_cache_map(CUtensorMap *map, const void *cache, int heads, int n_valid, int max_seq, bool fp16, int box_rows = kKN) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_valid, (cuuint64_t)heads};
     const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)max_seq * kHeadDim * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kKN, 1};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     return enc(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(cache), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

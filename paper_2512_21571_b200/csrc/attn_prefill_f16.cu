@@ -3,19 +3,18 @@
 // Same computation as attn_prefill_tc.cu (Section 3.1.2, Eq. 1: the score / probability tile stays on the SM between
 // the two products), for the case where Q, P and the cache rows travel as one fp16 term each.  The organisation differs:
 // a CTA is small enough (192 threads, 97 KB of shared memory, 256 tensor-memory columns) for two of them to share an SM,
-// and each one runs its chain  S = Q K_j^T  ->  softmax  ->  O += P_j V_j  strictly in order on ONE score buffer.  The
-// overlap of tensor-core work with softmax work comes from the other CTA of the SM, which also hides a CTA's set-up
-// (query load, norm, rotation) and its output pass behind the partner's steady state.
+// so that one CTA's set-up (query load, norm, rotation) and output pass hide behind the other's steady state, and the
+// cache is walked in steps of 64 positions with TWO score buffers of 64 columns: while the softmax warps work on step j
+// the tensor cores compute S_{j+1} = Q K_{j+1}^T and O += P_{j-1} V_{j-1}.
 //
-//   warp 0      TMA producer: K tile and V tile of 128 cache positions each (two 128B-swizzled boxes of 64
-//               head-dimension elements), single-buffered: K_{j+1} is requested when S_j is complete, V_{j+1} when
-//               O += P_j V_j is complete; both have a softmax pass of slack before they are needed.
+//   warp 0      TMA producer: K and V tiles of 64 cache positions (two 128B-swizzled boxes of 64 head-dimension
+//               elements each), two stages.
 //   warp 1      MMA issuer (one lane).  Q is a shared-memory operand here (tensor memory has no room for it beside
-//               S and O in half an SM's columns).
+//               two S buffers and O in half an SM's columns).
 //   warps 2-5   softmax, ONE thread per query row: no exchange between threads at all.  The thread loads its fp32
 //               query row (optionally applying the per-head RMSNorm and RoPE), scales it to log2 units and writes it to
-//               shared memory in the K-major swizzled operand layout; per tile: 128 scores -> mask (diagonal tiles) ->
-//               exp2 -> fp16 probabilities over the first 64 columns of S; finally O / l to the output.
+//               shared memory in the K-major swizzled operand layout; per step: 64 scores -> mask (diagonal tiles) ->
+//               exp2 -> fp16 probabilities over the first 32 columns of the step's S buffer; finally O / l to the output.
 // Online softmax with the lazy maximum of attn_prefill_tc.cu (threshold 2^8).  Every mbarrier wait is bounded; on
 // expiry the CTA raises the status word, drains and frees its tensor memory.
 #include "attn_prefill_common.cuh"
@@ -26,9 +25,17 @@ namespace {
 
 constexpr int kFThreads = 192;
 constexpr int kFSoftmax = 128;
-constexpr int kFSmem = 3 * kTile + 1024 /*align slack*/ + 128 /*barriers*/;   // Q, K, V
-constexpr uint32_t kFColS = 0, kFColO = 128, kFTmemCols = 256;
+constexpr int kStep = 64;                          // cache positions per step
+constexpr int kHalfSlab = kStep * 128;             // bytes of a [64 positions][64 x 16 bit] swizzled slab
+constexpr int kStepTile = 2 * kHalfSlab;           // [64][128] 16-bit tile
+constexpr int kFSmem = kTile + 4 * kStepTile + 1024 /*align slack*/ + 128 /*barriers*/;   // Q, 2 x (K, V)
+constexpr uint32_t kFColS = 0, kFColO = 128, kFTmemCols = 256;   // S buffers at columns 0 and 64
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -38,10 +45,16 @@ __global__ void __launch_bounds__(kFThreads, 2)
 attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_tile = base, k_tile = base + (uint32_t)kTile, v_tile = base + 2u * kTile;
-    const uint32_t bars = base + 3u * kTile;
-    const uint32_t q_ready = bars, k_full = bars + 8u, v_full = bars + 16u, s_full = bars + 24u, p_full = bars + 32u,
-                   pv_done = bars + 40u;
+    const uint32_t q_tile = base;
+    auto k_tile = [&](int st) { return base + (uint32_t)kTile + (uint32_t)st * 2u * kStepTile; };
+    auto v_tile = [&](int st) { return k_tile(st) + (uint32_t)kStepTile; };
+    const uint32_t bars = base + (uint32_t)kTile + 4u * kStepTile;
+    const uint32_t q_ready = bars;
+    auto k_full = [&](int st) { return bars + 8u * (1 + st); };
+    auto v_full = [&](int st) { return bars + 8u * (3 + st); };
+    auto s_full = [&](int st) { return bars + 8u * (5 + st); };
+    auto p_full = [&](int st) { return bars + 8u * (7 + st); };
+    auto pv_done = [&](int st) { return bars + 8u * (9 + st); };
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -65,15 +78,17 @@ attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int q0 = qt * kQM;
     const int n_valid = p.n_past + p.T;
     const int n_keys = min(p.n_past + q0 + kQM, n_valid);   // cache positions the last row of this tile may see
-    const int n_tiles = (n_keys + kKN - 1) / kKN;
+    const int n_tiles = (n_keys + kStep - 1) / kStep;   // steps of 64 cache positions
     const bool traced = NNC_TRACE_ALL_CTAS || (h == p.nq / 2 && seq == 0);   // tracing builds only
     (void)traced;
 
     if (threadIdx.x == 0) {
         abort_s = 0;
         mbar_init(q_ready, kFSoftmax);
-        mbar_init(k_full, 1); mbar_init(v_full, 1); mbar_init(s_full, 1);
-        mbar_init(p_full, kFSoftmax); mbar_init(pv_done, 1);
+        for (int st = 0; st < 2; ++st) {
+            mbar_init(k_full(st), 1); mbar_init(v_full(st), 1); mbar_init(s_full(st), 1);
+            mbar_init(p_full(st), kFSoftmax); mbar_init(pv_done(st), 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -93,50 +108,74 @@ attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (lane == 0) {   // ---------------- TMA producer ----------------
             pdl_wait();    // the cache rows of the new tokens come from the preceding kernel
             const int z = seq * p.nkv + jkv;
-            for (int j = 0; j < n_tiles; ++j) {
-                const uint32_t prev = (uint32_t)((j - 1) & 1);
-                if (j > 0 && !mbar_wait(s_full, prev, abort_flag, p.status, 31)) break;    // K_{j-1} has been read
-                mbar_expect_tx(k_full, kTile);
-                tma_load_3d(k_tile, &map_k, k_full, 0, j * kKN, z);
-                tma_load_3d(k_tile + kSlab, &map_k, k_full, 64, j * kKN, z);
-                if (j > 0 && !mbar_wait(pv_done, prev, abort_flag, p.status, 32)) break;   // V_{j-1} has been read
-                mbar_expect_tx(v_full, kTile);
-                tma_load_3d(v_tile, &map_v, v_full, 0, j * kKN, z);
-                tma_load_3d(v_tile + kSlab, &map_v, v_full, 64, j * kKN, z);
+            auto load_k = [&](int j) {
+                const int st = j & 1;
+                mbar_expect_tx(k_full(st), kStepTile);
+                tma_load_3d(k_tile(st), &map_k, k_full(st), 0, j * kStep, z);
+                tma_load_3d(k_tile(st) + kHalfSlab, &map_k, k_full(st), 64, j * kStep, z);
+            };
+            auto load_v = [&](int j) {
+                const int st = j & 1;
+                mbar_expect_tx(v_full(st), kStepTile);
+                tma_load_3d(v_tile(st), &map_v, v_full(st), 0, j * kStep, z);
+                tma_load_3d(v_tile(st) + kHalfSlab, &map_v, v_full(st), 64, j * kStep, z);
+            };
+            // A stage's K tile is free as soon as the S of the step that read it is complete -- a whole softmax pass before
+            // that step's second product -- so K runs one step ahead of V here: K_{j+1} is requested when S_{j-1} is
+            // complete, V_j when O += P_{j-2} V_{j-2} is.  The events come in exactly this order, and each load has more
+            // than a softmax pass before it is needed.
+            load_k(0);
+            if (n_tiles > 1) load_k(1);
+            load_v(0);
+            for (int j = 1; j < n_tiles; ++j) {
+                if (j + 1 < n_tiles) {
+                    if (!mbar_wait(s_full((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, p.status, 31)) break;
+                    load_k(j + 1);
+                }
+                if (j >= 2 && !mbar_wait(pv_done(j & 1), (uint32_t)(((j - 2) >> 1) & 1), abort_flag, p.status, 32)) break;
+                load_v(j);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc_qk = make_idesc(kKN, true, false);
+            constexpr uint32_t idesc_qk = make_idesc(kStep, true, false);
             constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true, true);
             bool ok = mbar_wait(q_ready, 0u, abort_flag, p.status, 33);
-            const uint64_t dq = make_smem_desc(q_tile), dk = make_smem_desc(k_tile);
-            const uint64_t dv = make_smem_desc_mn(v_tile, kSlab);
-            const uint32_t ts = tmem_base + kFColS, to = tmem_base + kFColO;
+            const uint64_t dq = make_smem_desc(q_tile);
+            const uint64_t dk[2] = {make_smem_desc(k_tile(0)), make_smem_desc(k_tile(1))};
+            const uint64_t dv[2] = {make_smem_desc_mn(v_tile(0), kHalfSlab), make_smem_desc_mn(v_tile(1), kHalfSlab)};
+            const uint32_t to = tmem_base + kFColO;
+            auto issue_qk = [&](int j) -> bool {
+                const int st = j & 1, u = j >> 1;
+                if (!mbar_wait(k_full(st), (uint32_t)(u & 1), abort_flag, p.status, 34)) return false;
+                // the score buffer holds P_{j-2} until O += P_{j-2} V_{j-2} has completed
+                if (j >= 2 && !mbar_wait(pv_done(st), (uint32_t)((u - 1) & 1), abort_flag, p.status, 35)) return false;
+                tc_fence_after();
+                const uint32_t d = tmem_base + kFColS + (uint32_t)st * kStep;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)     // 16 head-dimension elements per instruction
+                    umma_bf16(d, dq + (uint64_t)(((ks >> 2) * kSlab + (ks & 3) * 32) >> 4),
+                              dk[st] + (uint64_t)(((ks >> 2) * kHalfSlab + (ks & 3) * 32) >> 4), idesc_qk, ks != 0);
+                umma_commit(s_full(st));
+                return true;
+            };
+            if (ok) ok = issue_qk(0);
             for (int j = 0; ok && j < n_tiles; ++j) {
-                const uint32_t par = (uint32_t)(j & 1);
                 const unsigned long long tr0 = NNC_TRACE_NOW();
                 (void)tr0;
-                if (!mbar_wait(k_full, par, abort_flag, p.status, 34)) break;
-                // the score buffer holds P_{j-1} until O += P_{j-1} V_{j-1} has completed
-                if (j > 0 && !mbar_wait(pv_done, par ^ 1u, abort_flag, p.status, 35)) break;
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 head-dimension elements per instruction
-                    const uint64_t off = (uint64_t)(((ks >> 2) * kSlab + (ks & 3) * 32) >> 4);
-                    umma_bf16(ts, dq + off, dk + off, idesc_qk, ks != 0);
-                }
-                umma_commit(s_full);
+                if (j + 1 < n_tiles && !issue_qk(j + 1)) break;
+                const int st = j & 1, u = j >> 1;
                 const unsigned long long tr1 = NNC_TRACE_NOW();
                 (void)tr1;
-                if (!mbar_wait(p_full, par, abort_flag, p.status, 36)) break;
-                if (!mbar_wait(v_full, par, abort_flag, p.status, 37)) break;
+                if (!mbar_wait(p_full(st), (uint32_t)(u & 1), abort_flag, p.status, 36)) break;
+                if (!mbar_wait(v_full(st), (uint32_t)(u & 1), abort_flag, p.status, 37)) break;
                 tc_fence_after();
-                NNC_TS(j, 0, tr0); NNC_TS(j, 1, tr1); NNC_TS(j, 2, NNC_TRACE_NOW());
+                if (j < 31) { NNC_TS(j, 0, tr0); NNC_TS(j, 1, tr1); NNC_TS(j, 2, NNC_TRACE_NOW()); }
+                const uint32_t pa = tmem_base + kFColS + (uint32_t)st * kStep;   // P: two positions per column
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)     // 16 cache positions per instruction; P: two positions per column
-                    umma_bf16_ts(to, ts + (uint32_t)ks * 8u, dv + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (j != 0) || (ks != 0));
-                umma_commit(pv_done);
+                for (int ks = 0; ks < 4; ++ks)     // 16 cache positions per instruction
+                    umma_bf16_ts(to, pa + (uint32_t)ks * 8u, dv[st] + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (j != 0) || (ks != 0));
+                umma_commit(pv_done(st));
             }
         }
     } else {   // ---------------- softmax warps 2..5: one thread per query row ----------------
@@ -186,50 +225,55 @@ attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             mbar_arrive(q_ready);
         }
         float m_used = -INFINITY, l = 0.f;
-        const uint32_t ts = tmem_base + lane_addr + kFColS, to = tmem_base + lane_addr + kFColO;
+        const uint32_t to = tmem_base + lane_addr + kFColO;
         bool ok = true;
         const unsigned long long tr_q = NNC_TRACE_NOW();
         (void)tr_q;
         for (int j = 0; j < n_tiles; ++j) {
+            const int st = j & 1, u = j >> 1;
             const unsigned long long ts0 = NNC_TRACE_NOW();
             (void)ts0;
-            ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)(j & 1), abort_flag, p.status, 38));
+            ok = __all_sync(0xffffffffu, mbar_wait(s_full(st), (uint32_t)(u & 1), abort_flag, p.status, 38));
             if (!ok) break;
             const unsigned long long ts1 = NNC_TRACE_NOW();
             (void)ts1;
             tc_fence_after();
-            // S_j complete also means O += P_{j-1} V_{j-1} is complete: the issuer waited for it before this product
-            uint32_t sv[4][32];
+            const uint32_t ts = tmem_base + lane_addr + kFColS + (uint32_t)st * kStep;
+            uint32_t sv[2][32];
             tmem_ld32_nowait(ts, sv[0]);
             tmem_ld32_nowait(ts + 32u, sv[1]);
-            tmem_ld32_nowait(ts + 64u, sv[2]);
-            tmem_ld32_nowait(ts + 96u, sv[3]);
             tmem_wait_ld();
             const unsigned long long ts2 = NNC_TRACE_NOW();
             (void)ts2;
-            if (j * kKN + kKN - 1 > p.n_past + q0) {   // the tile reaches past the first row's position: causal mask
-                const int k0 = j * kKN;
+            if (j * kStep + kStep - 1 > p.n_past + q0) {   // the step reaches past the first row's position: causal mask
+                const int k0 = j * kStep;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
                         if (k0 + 32 * c + e > pos) sv[c][e] = 0xff800000u;   // -inf
             }
+            // three-input maxima, four independent chains
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    mx[0] = fmaxf(mx[0], __uint_as_float(sv[c][e]));     mx[1] = fmaxf(mx[1], __uint_as_float(sv[c][e + 1]));
-                    mx[2] = fmaxf(mx[2], __uint_as_float(sv[c][e + 2])); mx[3] = fmaxf(mx[3], __uint_as_float(sv[c][e + 3]));
+                for (int e = 0; e < 32; e += 8) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) mx[q] = max3(mx[q], __uint_as_float(sv[c][e + 2 * q]), __uint_as_float(sv[c][e + 2 * q + 1]));
                 }
             const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             if (j == 0) {
                 m_used = m_tile;   // finite: position 0 is visible to every row
             } else {
+                // a row whose step is masked out entirely (the second half of a diagonal tile) has m_tile = -inf: no move
                 const bool need = m_tile > m_used + kLazyMax;
                 if (__any_sync(0xffffffffu, need)) {
-                    // O is rescaled in tensor memory, 32 columns at a time; rows that keep their maximum multiply by 1
+                    // O is rescaled in tensor memory, 32 columns at a time; rows that keep their maximum multiply by 1.
+                    // The product of the previous step must have landed first.
+                    ok = __all_sync(0xffffffffu, mbar_wait(pv_done((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, p.status, 40));
+                    if (!ok) break;
+                    tc_fence_after();
                     const float m_new = need ? m_tile : m_used;
                     const float alpha = ex2_approx(m_used - m_new);
 #pragma unroll 1
@@ -247,34 +291,35 @@ attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             }
             // exponents are <= 2^8 by the lazy maximum; results below 2^-126 flush to zero, which a row sum >= 1 cannot see.
             // P over S: fp16 pairs, two positions per column, so chunk c (positions 32 c .. 32 c + 31) lands in columns
-            // 16 c .. 16 c + 15 -- columns whose scores this thread already holds in registers.
-            float sum[4] = {0.f, 0.f, 0.f, 0.f};
+            // 16 c .. 16 c + 15 of the step's buffer -- columns whose scores this thread already holds in registers.
+            // the subtraction and the row sum run as packed two-lane fp32 operations: half the instructions
+            float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            const float2 neg_m = make_float2(-m_used, -m_used);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t ph[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float a = ex2_approx(__uint_as_float(sv[c][2 * e]) - m_used);
-                    const float b = ex2_approx(__uint_as_float(sv[c][2 * e + 1]) - m_used);
-                    sum[(2 * e) & 3] += a;
-                    sum[(2 * e + 1) & 3] += b;
-                    ph[e] = pack_f16x2_sat(a, b);   // probabilities are at most 2^8: inside the fp16 range
+                    const float2 x = __fadd2_rn(make_float2(__uint_as_float(sv[c][2 * e]), __uint_as_float(sv[c][2 * e + 1])), neg_m);
+                    const float2 pr = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                    sum[e & 1] = __fadd2_rn(sum[e & 1], pr);
+                    ph[e] = pack_f16x2_sat(pr.x, pr.y);   // probabilities are at most 2^8: inside the fp16 range
                 }
                 tmem_st16(ts + 16u * c, ph);
             }
-            l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            l += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
             const unsigned long long ts3 = NNC_TRACE_NOW();
             (void)ts3;
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(p_full);
-            if (warp == 2 && lane == 0) { NNC_TS(j, 3, ts0); NNC_TS(j, 4, ts1); NNC_TS(j, 5, ts2); NNC_TS(j, 6, ts3); NNC_TS(j, 7, NNC_TRACE_NOW()); }
+            mbar_arrive(p_full(st));
+            if (warp == 2 && lane == 0 && j < 31) { NNC_TS(j, 3, ts0); NNC_TS(j, 4, ts1); NNC_TS(j, 5, ts2); NNC_TS(j, 6, ts3); NNC_TS(j, 7, NNC_TRACE_NOW()); }
         }
         // ---- O / l -> output ----
         const unsigned long long tr_e = NNC_TRACE_NOW();
         (void)tr_e;
         if (warp == 2 && lane == 0) { NNC_TS(31, 0, tr_q); NNC_TS(31, 1, tr_e); }
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done, (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status, 39));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done((n_tiles - 1) & 1), (uint32_t)(((n_tiles - 1) >> 1) & 1), abort_flag, p.status, 39));
         if (ok) {
             tc_fence_after();
             const float inv = 1.f / l;

@@ -13,8 +13,8 @@
 //   warp 1      MMA issuer (one lane): S[j&1] = Q K_j^T into one of two score buffers, so the product of tile j+1
 //               runs while the softmax warps work on tile j; then O += P_j V_j with V as an MN-major operand (the
 //               cache row is [position][head dim], contraction over positions).  Q, like P, is an A operand in
-//               TENSOR memory: a 128 x 128 x 16 instruction with both operands in shared memory would read 8 KB per
-//               64 cycles, all the shared-memory bandwidth an SM has; with A in tensor memory only K or V moves.
+//               TENSOR memory, which leaves the shared memory to K and V (a 128 x 128 x 16 instruction issues every
+//               ~65 cycles with A in either place).
 //   warps 2-9   softmax: two threads per query row (warps w and w + 4 share a tensor-memory lane quarter and split
 //               the 128 columns of a row between them; the row maximum crosses through shared memory).  They load Q
 //               (fp32; optionally applying the per-head RMSNorm and RoPE on the way: a thread holds the whole head, so
@@ -42,9 +42,8 @@ constexpr int kPfSmem = 4 * kTile + 1024 /*align slack*/ + 256 /*barriers*/;   /
 constexpr uint32_t kColS = 0, kColO = 256, kColQ = 384, kTmemCols = 512;
 
 // OUT_FP16: the output is one fp16 matrix (saturating) instead of a bf16 value + residual pair.
-// F16: the tensor maps cover an fp16 image of the K/V rows (exact for bf16 values inside the fp16 range), and Q and P
-// travel as ONE fp16 term each: half the tensor-core instructions of the two-bf16-term form.
-template <bool OUT_FP16, bool F16>
+// (The one-term fp16 form of the same computation is a kernel of its own, attn_prefill_f16.cu.)
+template <bool OUT_FP16>
 __global__ void __launch_bounds__(kPfThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -114,13 +113,13 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc_qk = make_idesc(kKN, F16, false);
-            constexpr uint32_t idesc_pv = make_idesc(kHeadDim, F16, true);
+            constexpr uint32_t idesc_qk = make_idesc(kKN, false, false);
+            constexpr uint32_t idesc_pv = make_idesc(kHeadDim, false, true);
             bool ok = mbar_wait(q_ready, 0u, abort_flag, p.status, 22);
             tc_fence_after();
             // Descriptors differ only in their 14-bit start-address field (bytes >> 4), so every operand descriptor of
             // the kernel is a base computed once plus a compile-time constant: the issuing thread spends a handful of
-            // instructions per tcgen05.mma, less than the 64 cycles one 128 x 128 x 16 instruction executes for.
+            // instructions per tcgen05.mma, less than the ~65 cycles one 128 x 128 x 16 instruction executes for.
             const uint32_t tq = tmem_base + kColQ;
             const uint64_t dk[2] = {make_smem_desc(k_tile(0)), make_smem_desc(k_tile(1))};
             const uint64_t dv[2] = {make_smem_desc_mn(v_tile(0), kSlab), make_smem_desc_mn(v_tile(1), kSlab)};
@@ -135,7 +134,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dimension elements per instruction
                     const uint64_t off = (uint64_t)(((ks >> 2) * kSlab + (ks & 3) * 32) >> 4);
                     umma_bf16_ts(d, tq + (uint32_t)ks * 8u, b0 + off, idesc_qk, ks != 0);
-                    if (!F16) umma_bf16_ts(d, tq + 64u + (uint32_t)ks * 8u, b0 + off, idesc_qk, 1u);
+                    umma_bf16_ts(d, tq + 64u + (uint32_t)ks * 8u, b0 + off, idesc_qk, 1u);
                 }
                 umma_commit(s_full(s));
                 return true;
@@ -157,7 +156,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int ks = 0; ks < 8; ++ks) {   // 16 cache positions per instruction
                     const uint64_t b = dv[s] + (uint64_t)(ks * (2048 >> 4));
                     umma_bf16_ts(d, pa + (uint32_t)ks * 8u, b, idesc_pv, (j != 0) || (ks != 0));
-                    if (!F16) umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
+                    umma_bf16_ts(d, pa + 64u + (uint32_t)ks * 8u, b, idesc_pv, 1u);
                 }
                 umma_commit(pv_done(s));
                 if (blockIdx.x == 0) NNC_TRACE_EVENT(302, tr0, tr1, NNC_TRACE_NOW());
@@ -210,16 +209,11 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 for (int e = 0; e < 16; ++e) {   // compile-time indices on both sides keep q[] in registers; half is warp-uniform
                     const float a = valid ? (half ? q[64 + 32 * i + 2 * e] : q[32 * i + 2 * e]) * qscale : 0.f;
                     const float b = valid ? (half ? q[64 + 32 * i + 2 * e + 1] : q[32 * i + 2 * e + 1]) * qscale : 0.f;
-                    if (F16) {
-                        qh[e] = pack_f16x2_sat(a, b);
-                        ql[e] = 0u;
-                    } else {
-                        qh[e] = pack_bf16x2(a, b);
-                        ql[e] = pack_bf16x2(a - bf16_lo(qh[e]), b - bf16_hi(qh[e]));
-                    }
+                    qh[e] = pack_bf16x2(a, b);
+                    ql[e] = pack_bf16x2(a - bf16_lo(qh[e]), b - bf16_hi(qh[e]));
                 }
                 tmem_st16(tqw + 16u * i, qh);
-                if (!F16) tmem_st16(tqw + 64u + 16u * i, ql);
+                tmem_st16(tqw + 64u + 16u * i, ql);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -313,22 +307,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
                 uint32_t ph[16], pl[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    if (F16) {   // probabilities are at most 2^8: inside the fp16 range
-                        ph[e] = pack_f16x2_sat(sv[32 * i + 2 * e], sv[32 * i + 2 * e + 1]);
-                        pl[e] = 0u;
-                    } else {
-                        // value = the upper 16 bits of the fp32 pattern (truncation), residual = the upper 16 bits of
-                        // what is left: byte permutes and two subtractions, nothing on the conversion pipe, which the
-                        // exponentials keep busy.  value + residual still carries 15-16 bits of the probability.
-                        const uint32_t a = __float_as_uint(sv[32 * i + 2 * e]), b = __float_as_uint(sv[32 * i + 2 * e + 1]);
-                        ph[e] = __byte_perm(a, b, 0x7632);
-                        const float ra = __uint_as_float(a) - __uint_as_float(a & 0xffff0000u);
-                        const float rb = __uint_as_float(b) - __uint_as_float(b & 0xffff0000u);
-                        pl[e] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
-                    }
+                    // value = the upper 16 bits of the fp32 pattern (truncation), residual = the upper 16 bits of
+                    // what is left: byte permutes and two subtractions, nothing on the conversion pipe, which the
+                    // exponentials keep busy.  value + residual still carries 15-16 bits of the probability.
+                    const uint32_t a = __float_as_uint(sv[32 * i + 2 * e]), b = __float_as_uint(sv[32 * i + 2 * e + 1]);
+                    ph[e] = __byte_perm(a, b, 0x7632);
+                    const float ra = __uint_as_float(a) - __uint_as_float(a & 0xffff0000u);
+                    const float rb = __uint_as_float(b) - __uint_as_float(b & 0xffff0000u);
+                    pl[e] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
                 }
                 tmem_st16(ts + 32u * half + 16u * i, ph);
-                if (!F16) tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
+                tmem_st16(ts + 64u + 32u * half + 16u * i, pl);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -394,9 +383,9 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
     }
 }
 
-template <bool OUT_FP16, bool F16>
+template <bool OUT_FP16>
 cudaError_t launch_pf(const LaunchCtx &lc, const CUtensorMap &mk, const CUtensorMap &mv, const PfParams &p, dim3 grid) {
-    auto kern = attn_prefill_tc_kernel<OUT_FP16, F16>;
+    auto kern = attn_prefill_tc_kernel<OUT_FP16>;
     static unsigned long long attr_done = 0;   // per instantiation, one bit per device
     if (cudaError_t e = ensure_dynamic_smem(kern, kPfSmem, &attr_done); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -425,8 +414,9 @@ cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows,
     if (T <= 0 || batch <= 0 || n_past < 0 || n_past + T > max_seq || nq % nkv) return cudaErrorInvalidValue;
     if (((uintptr_t)qkv | (uintptr_t)kcache | (uintptr_t)vcache | (uintptr_t)out | (uintptr_t)out_lo) & 15) return cudaErrorInvalidValue;
     CUtensorMap mk, mv;
-    if (!make_cache_map(&mk, kcache, batch * nkv, n_past + T, max_seq, kv_f16) ||
-        !make_cache_map(&mv, vcache, batch * nkv, n_past + T, max_seq, kv_f16))
+    const int box_rows = kv_f16 ? 64 : kKN;   // the fp16 form walks the cache in steps of 64 positions
+    if (!make_cache_map(&mk, kcache, batch * nkv, n_past + T, max_seq, kv_f16, box_rows) ||
+        !make_cache_map(&mv, vcache, batch * nkv, n_past + T, max_seq, kv_f16, box_rows))
         return cudaErrorInvalidValue;
     PfParams p;
     p.qkv = qkv; p.row_stride = (nq + 2 * nkv) * kHeadDim; p.out = out; p.out_lo = out_lo;
@@ -435,7 +425,7 @@ cudaError_t launch_attn_prefill(const LaunchCtx &lc, const float *qkv, int rows,
     p.batch = batch; p.n_qt = (T + kQM - 1) / kQM;
     const dim3 grid((unsigned)(p.n_qt * nq * batch));
     if (kv_f16) return launch_attn_prefill_f16(lc, mk, mv, p, grid, out_fp16);
-    return out_fp16 ? launch_pf<true, false>(lc, mk, mv, p, grid) : launch_pf<false, false>(lc, mk, mv, p, grid);
+    return out_fp16 ? launch_pf<true>(lc, mk, mv, p, grid) : launch_pf<false>(lc, mk, mv, p, grid);
 }
 
 }  // namespace nnc

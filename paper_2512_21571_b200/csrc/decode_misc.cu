@@ -97,6 +97,7 @@ __global__ void __launch_bounds__(256)
 rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, bf16 *__restrict__ out,
                     bf16 *__restrict__ out_lo, int H, float eps, int first, int step) {
     __shared__ float red[8];
+    NNC_TRACE_SCOPE(4);
     pdl_launch_dependents();   // the next kernel may set itself up while this one runs
     pdl_wait();
     const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);

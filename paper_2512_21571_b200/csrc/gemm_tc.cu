@@ -90,14 +90,13 @@ struct WorkIter {
 
 // Shared-memory stage: [weight tile][activation tile][activation residual tile (SPLIT)].
 // SWAP puts the weights on the M side (128 rows) and BN tokens on the N side; otherwise 128 tokens x BN weights.
-// CPS: CTAs meant to share an SM (1 or 2); two get half of the shared memory each.
-template <int BN, bool SWAP, bool SPLIT, int KA, int CPS = 1>
+template <int BN, bool SWAP, bool SPLIT, int KA>
 struct SmemLayout {
     static constexpr int kW = (SWAP ? kBM : BN) * kBK * 2;
     static constexpr int kX = (SWAP ? BN : kBM) * kBK * 2;
     static constexpr int kAtom = kW + kX * (SPLIT ? 2 : 1);   // one 64-wide K slab of every operand
     static constexpr int kStage = KA * kAtom;                 // KA slabs per pipeline stage
-    static constexpr int kStagesFit = ((CPS == 2 ? 96 : 192) * 1024) / kStage;
+    static constexpr int kStagesFit = (192 * 1024) / kStage;
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr int kBytes = kStages * kStage + 1024 /*align slack*/ + 256 /*barriers*/;
     static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
@@ -109,16 +108,11 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + 
 // SPLIT: the activations come as two bf16 matrices (value and rounding residual); both are multiplied with the
 // same weight tile into the same accumulator, which restores ~16 mantissa bits on the activation side.
 // F16: operands are fp16 (single term) and the SwiGLU epilogue writes one fp16 matrix (saturating at +-65504).
-// CPS = 2 (few-token form): the grid is two CTAs per SM, each with half of the ring.  While one of them parks or
-// collects partial tiles and runs its epilogue the other keeps streaming, and the CTAs of the next kernel in the stream
-// (launched programmatically) move in as soon as ONE of this kernel's CTAs on an SM has left, and request their first
-// weight tiles while this kernel is still finishing.
-template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16, int CPS>
-__global__ void __launch_bounds__(kGemmThreads, CPS)
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16>
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_x_lo, GemmParams p) {
-    using L = SmemLayout<BN, SWAP, SPLIT, KA, CPS>;
-    static_assert(L::kStages >= 2, "the ring needs two stages");
+    using L = SmemLayout<BN, SWAP, SPLIT, KA>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = base + L::kStages * L::kStage;      // full[S], empty[S], tfull[2], tempty[2], 8 B each
@@ -161,26 +155,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {  // ---------------- TMA producer ----------------
-            // The weights are never written by a kernel of the same stream, so the ring's first pass of weight tiles is
-            // requested before the wait for the previous kernel: it streams in while that kernel finishes.  The
-            // activation tiles of those stages follow after the wait and complete the same stage barriers.
-            int early = 0;
-            {
-                WorkIter itw(total_tiles, kb_count, stream);
-                Segment gw;
-                while (early < L::kStages && itw.next(gw)) {
-                    const int w_row = SWAP ? (gw.tile_id % p.m_tiles) * kBM : (gw.tile_id / p.m_tiles) * BN;
-                    for (int kb = gw.kb_lo; kb < gw.kb_hi && early < L::kStages; ++kb, ++early) {
-                        mbar_expect_tx(full_bar(early), L::kStage);
-                        const uint32_t sw = base + early * L::kStage;
-#pragma unroll
-                        for (int a = 0; a < KA; ++a)
-                            tma_load_2d(sw + a * L::kAtom, &map_w, full_bar(early), (kb * KA + a) * kBK, w_row);
-                    }
-                }
-            }
             pdl_wait();
-            int stage = 0, unit = 0;
+            int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             WorkIter it(total_tiles, kb_count, stream);
@@ -193,18 +169,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const unsigned long long tr0 = NNC_TRACE_NOW();
                 (void)tr0;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
-                    const bool w_here = unit >= early;   // else this stage's weights are already on their way
-                    ++unit;
-                    if (w_here) {
-                        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(stage), L::kStage);
-                    }
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(stage), L::kStage);
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
                     for (int a = 0; a < KA; ++a) {   // KA consecutive slabs: KA * 128 contiguous bytes of every weight row
                         const uint32_t sa = sw + a * L::kAtom;
                         const int kx = (kb * KA + a) * kBK;
-                        if (w_here) tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
+                        tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
                         tma_load_2d(sa + L::kW, &map_x, full_bar(stage), kx, x_row);
                         if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage), kx, x_row);
                     }
@@ -421,14 +393,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             float sum[32];
 #pragma unroll
                             for (int i = 0; i < 32; ++i) sum[i] = __uint_as_float(r[i]);
-                            // the parked pieces are added in K order; up to kU pieces' loads are in flight at a time (fewer under the
-                            // register limit of two CTAs per SM)
-                            constexpr int kU = CPS == 2 ? 2 : 4;
+                            // the parked pieces are added in K order; up to four pieces' loads are in flight at a time
                             const size_t in_slot = ((size_t)(c0 >> 5) * 8 * kBM + row) * 4;
-                            for (int q0 = 1; q0 < g.n_pieces; q0 += kU) {
-                                float4 v[kU][8];
+                            for (int q0 = 1; q0 < g.n_pieces; q0 += 4) {
+                                float4 v[4][8];
 #pragma unroll
-                                for (int u = 0; u < kU; ++u) {
+                                for (int u = 0; u < 4; ++u) {
                                     if (q0 + u < g.n_pieces) {
                                         const float4 *src = reinterpret_cast<const float4 *>(
                                             p.part + (size_t)it.slot_of(g.first_cta + q0 + u, tile_id) * kSlotFloats + in_slot);
@@ -437,7 +407,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                     }
                                 }
 #pragma unroll
-                                for (int u = 0; u < kU; ++u) {
+                                for (int u = 0; u < 4; ++u) {
                                     if (q0 + u < g.n_pieces) {
 #pragma unroll
                                         for (int i = 0; i < 8; ++i) {
@@ -597,11 +567,11 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int K, int box_rows, 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16 = false, int CPS = 1>
+template <int BN, bool SWAP, int EPI, bool SPLIT, int KA, bool F16 = false>
 cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
                       int K, int ldy, int *status, const GemmScratch *scratch, const float *out_scale = nullptr) {
-    using L = SmemLayout<BN, SWAP, SPLIT, KA, CPS>;
-    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA, F16, CPS>;
+    using L = SmemLayout<BN, SWAP, SPLIT, KA>;
+    auto kern = gemm_tc_kernel<BN, SWAP, EPI, SPLIT, KA, F16>;
     static unsigned long long attr_done = 0;   // per instantiation, one bit per device
     if (cudaError_t e = ensure_dynamic_smem(kern, L::kBytes, &attr_done); e != cudaSuccess) return e;
     CUtensorMap map_w, map_x, map_x_lo;
@@ -622,16 +592,13 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
     // equal contiguous range per CTA instead; tiles that straddle a cut are finished through partial tiles in scratch.
     p.stream = 0; p.part = nullptr; p.tickets = nullptr; p.part_bytes = 0;
     const int tiles = p.m_tiles * p.n_tiles;
-    int grid = tiles < CPS * lc.sm_count ? tiles : CPS * lc.sm_count;
+    int grid = tiles < lc.sm_count ? tiles : lc.sm_count;
     if (SWAP && scratch && scratch->part && scratch->tickets) {
         const long long stages = (long long)tiles * (K / (kBK * KA));
-        // two CTAs per SM only when every CTA still gets six stages or more; otherwise one half-size CTA per SM, which
-        // leaves the other half of the SM to the next kernel's CTAs
-        const int slots = (CPS == 2 && stages >= 12ll * lc.sm_count) ? 2 * lc.sm_count : lc.sm_count;
-        const int g = stages < slots ? (int)stages : slots;
+        const int g = stages < lc.sm_count ? (int)stages : lc.sm_count;
         const double whole_tile_eff = (double)tiles / (((tiles + lc.sm_count - 1) / lc.sm_count) * (double)lc.sm_count);
         const size_t need = (size_t)2 * g * BN * kBM * sizeof(float);
-        if ((CPS == 2 || whole_tile_eff < 0.97) && need <= scratch->part_bytes && 2 * g <= scratch->n_tickets) {
+        if (whole_tile_eff < 0.97 && need <= scratch->part_bytes && 2 * g <= scratch->n_tickets) {
             p.stream = 1; p.part = scratch->part; p.tickets = scratch->tickets; p.part_bytes = scratch->part_bytes;
             grid = g;
         }
@@ -656,9 +623,6 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
 template <int BN, bool SWAP, int EPI, bool SPLIT>
 cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
                       int K, int ldy, int *status, const GemmScratch *scratch) {
-    // <= 32 tokens: half-size CTAs (two fit an SM), two K slabs per stage, unless the product is tiny
-    if (SWAP && BN == 32 && K % (2 * kBK) == 0 && scratch && (long long)((N + kBM - 1) / kBM) * (K / (2 * kBK)) >= 4ll * lc.sm_count)
-        return launch_tc_ka<BN, SWAP, EPI, SPLIT, (SWAP && BN == 32) ? 2 : 1, false, (SWAP && BN == 32) ? 2 : 1>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, scratch);
     if (SWAP && BN == 32 && K % (4 * kBK) == 0)
         return launch_tc_ka<BN, SWAP, EPI, SPLIT, (SWAP && BN == 32) ? 4 : 1>(lc, X, X_lo, W, Y, Y_lo, T, N, K, ldy, status, scratch);
     if (SWAP && BN == 64 && K % (2 * kBK) == 0)
