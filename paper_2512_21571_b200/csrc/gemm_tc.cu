@@ -115,11 +115,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     using L = SmemLayout<BN, SWAP, SPLIT, KA>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = base + L::kStages * L::kStage;      // full[S], empty[S], tfull[2], tempty[2], 8 B each
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (L::kStages + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * L::kStages + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * L::kStages + 2 + a); };
+    const uint32_t bars = base + L::kStages * L::kStage;      // full[S][KA], empty[S], tfull[2], tempty[2], 8 B each
+    // full: one barrier per K slab of a stage, so that the MMAs of a stage start when its FIRST slab has landed (a stage of
+    // four slabs is 96 KB; waiting for all of it would cost the start of every product a microsecond or two)
+    static_assert((L::kStages * (KA + 1) + 4) * 8 <= 256, "barrier block");
+    auto full_bar = [&](int s, int a) { return bars + 8u * (s * KA + a); };
+    auto empty_bar = [&](int s) { return bars + 8u * (L::kStages * KA + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (L::kStages * (KA + 1) + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (L::kStages * (KA + 1) + 2 + a); };
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ bool split_last;
@@ -130,7 +133,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (threadIdx.x == 0) {
         abort_s = 0;
-        for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < L::kStages; ++s) {
+            for (int a = 0; a < KA; ++a) mbar_init(full_bar(s, a), 1);
+            mbar_init(empty_bar(s), 1);
+        }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -170,15 +176,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 (void)tr0;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(stage), L::kStage);
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
                     for (int a = 0; a < KA; ++a) {   // KA consecutive slabs: KA * 128 contiguous bytes of every weight row
                         const uint32_t sa = sw + a * L::kAtom;
                         const int kx = (kb * KA + a) * kBK;
-                        tma_load_2d(sa, &map_w, full_bar(stage), kx, w_row);
-                        tma_load_2d(sa + L::kW, &map_x, full_bar(stage), kx, x_row);
-                        if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage), kx, x_row);
+                        mbar_expect_tx(full_bar(stage, a), L::kAtom);
+                        tma_load_2d(sa, &map_w, full_bar(stage, a), kx, w_row);
+                        tma_load_2d(sa + L::kW, &map_x, full_bar(stage, a), kx, x_row);
+                        if (SPLIT) tma_load_2d(sa + L::kW + L::kX, &map_x_lo, full_bar(stage, a), kx, x_row);
                     }
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -202,12 +208,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 (void)tr0; (void)tr_first;
                 const int kb_lo = g.kb_lo, kb_hi = g.kb_hi;
                 for (int kb = kb_lo; kb < kb_hi; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
-                    if (kb == kb_lo) tr_first = NNC_TRACE_NOW();
-                    tc_fence_after();
                     const uint32_t sw = base + stage * L::kStage;
 #pragma unroll
                     for (int a = 0; a < KA; ++a) {
+                        if (!mbar_wait(full_bar(stage, a), phase, abort_flag, p.status, 3)) { ok = false; break; }
+                        if (kb == kb_lo && a == 0) tr_first = NNC_TRACE_NOW();
+                        tc_fence_after();
                         const uint32_t sa = sw + a * L::kAtom;
                         const uint64_t dw = make_smem_desc(sa), dx = make_smem_desc(sa + L::kW),
                                        dxl = make_smem_desc(sa + L::kW + L::kX);
@@ -224,6 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             }
                         }
                     }
+                    if (!ok) break;
                     umma_commit(empty_bar(stage));
                     if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -355,6 +362,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(203, tr0, tr1, NNC_TRACE_NOW());
                 } else {
+                    // Accumulating epilogue of a 32-token tile: the old output values do not depend on the other pieces, so
+                    // they are requested now and arrive while this CTA waits for the flags and reads the pieces.
+                    constexpr bool kOldEarly = EPI == 2 && BN == 32;
+                    float old_y[kOldEarly ? 32 : 1];
+                    if (kOldEarly && got) {
+                        const float *y = reinterpret_cast<const float *>(p.Y) + m;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            old_y[i] = (m < p.N && nt * BN + i < p.T) ? __ldcg(y + (size_t)(nt * BN + i) * p.ldy) : 0.f;
+                    }
                     if (warp == 2) {
                         // bounded wait for the other pieces (they never wait for anything of this CTA's); one flag per
                         // lane, so that all of them are polled in one memory round trip
@@ -393,12 +410,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             float sum[32];
 #pragma unroll
                             for (int i = 0; i < 32; ++i) sum[i] = __uint_as_float(r[i]);
-                            // the parked pieces are added in K order; up to four pieces' loads are in flight at a time
+                            // the parked pieces are added in K order; up to kU pieces' loads are in flight at a time
+                            constexpr int kU = kOldEarly ? 3 : 4;   // the early old values take a piece's worth of registers
                             const size_t in_slot = ((size_t)(c0 >> 5) * 8 * kBM + row) * 4;
-                            for (int q0 = 1; q0 < g.n_pieces; q0 += 4) {
-                                float4 v[4][8];
+                            for (int q0 = 1; q0 < g.n_pieces; q0 += kU) {
+                                float4 v[kU][8];
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) {
+                                for (int u = 0; u < kU; ++u) {
                                     if (q0 + u < g.n_pieces) {
                                         const float4 *src = reinterpret_cast<const float4 *>(
                                             p.part + (size_t)it.slot_of(g.first_cta + q0 + u, tile_id) * kSlotFloats + in_slot);
@@ -407,7 +425,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                     }
                                 }
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) {
+                                for (int u = 0; u < kU; ++u) {
                                     if (q0 + u < g.n_pieces) {
 #pragma unroll
                                         for (int i = 0; i < 8; ++i) {
@@ -421,7 +439,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[i] * osc);
                             const unsigned long long tr2 = NNC_TRACE_NOW();
                             (void)tr2;
-                            store_swap(r, m, nt * BN + c0);
+                            if (kOldEarly) {
+                                float *y = reinterpret_cast<float *>(p.Y) + m;
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (m < p.N && nt * BN + i < p.T) y[(size_t)(nt * BN + i) * p.ldy] = old_y[i] + __uint_as_float(r[i]);
+                            } else {
+                                store_swap(r, m, nt * BN + c0);
+                            }
                             if ((NNC_TRACE_ALL_CTAS || blockIdx.x == 0) && warp == 2 && lane == 0) NNC_TRACE_EVENT(206, tr1, tr2, NNC_TRACE_NOW());
                         }
                     }
