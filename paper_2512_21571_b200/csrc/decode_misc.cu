@@ -99,13 +99,20 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
     __shared__ float red[8];
     NNC_TRACE_SCOPE(4);
     pdl_launch_dependents();   // the next kernel may set itself up while this one runs
-    pdl_wait();
-    const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
-    uint2 *dst = reinterpret_cast<uint2 *>(out + (size_t)blockIdx.x * H);
     // rows of up to 4096 elements stay in registers between the two passes (4 x 16 bytes per thread, all requested
     // at once); longer rows are read again
     constexpr int kKeep = 4;
     const int n4 = H / 4;
+    // the gains are weights: they are requested before the wait for the kernel that produces x
+    uint2 gk[kKeep];
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const int i = threadIdx.x + 256 * u;
+        gk[u] = (i < n4) ? reinterpret_cast<const uint2 *>(gain)[i] : make_uint2(0u, 0u);
+    }
+    pdl_wait();
+    const float4 *src = reinterpret_cast<const float4 *>(x + (size_t)(first + blockIdx.x * step) * H);
+    uint2 *dst = reinterpret_cast<uint2 *>(out + (size_t)blockIdx.x * H);
     float4 keep[kKeep];
     float ss = 0.f;
 #pragma unroll
@@ -126,8 +133,7 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)H + eps);
-    auto emit = [&](int i, const float4 &v) {
-        const uint2 g = reinterpret_cast<const uint2 *>(gain)[i];
+    auto emit = [&](int i, const float4 &v, const uint2 g) {
         const float y0 = v.x * inv * bf16_lo(g.x), y1 = v.y * inv * bf16_hi(g.x);
         const float y2 = v.z * inv * bf16_lo(g.y), y3 = v.w * inv * bf16_hi(g.y);
         uint2 o;
@@ -150,9 +156,9 @@ rmsnorm_rows_kernel(const float *__restrict__ x, const bf16 *__restrict__ gain, 
 #pragma unroll
     for (int u = 0; u < kKeep; ++u) {
         const int i = threadIdx.x + 256 * u;
-        if (i < n4) emit(i, keep[u]);
+        if (i < n4) emit(i, keep[u], gk[u]);
     }
-    for (int i = threadIdx.x + 256 * kKeep; i < n4; i += 256) emit(i, src[i]);
+    for (int i = threadIdx.x + 256 * kKeep; i < n4; i += 256) emit(i, src[i], reinterpret_cast<const uint2 *>(gain)[i]);
 }
 
 // dst[h][pos][:] = fp16(src[h][pos][:]) for pos < n_pos; 16 bytes (8 elements) per thread
