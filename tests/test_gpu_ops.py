@@ -276,7 +276,8 @@ def test_gemm_f16_against_oracle(nnc, oracle_mod, T, N, K):
     (1, 19, 2, 1, 0, 0.0), (2, 130, 4, 2, 7, 0.0), (1, 300, 8, 2, 0, 0.0), (1, 64, 16, 8, 200, 0.0),
     (1, 128, 1, 1, 0, 0.0), (1, 129, 2, 2, 127, 0.0),            # exactly one tile; one row past a tile boundary
     (1, 2048, 4, 1, 100, 0.0),                                    # the prompt length of the batched workload, with a past
-    (1, 700, 2, 1, 60, 0.15), (1, 400, 2, 2, 0, 1.0)])            # keys that grow along the sequence: the running maximum moves
+    (1, 700, 2, 1, 60, 0.15), (1, 400, 2, 2, 0, 1.0),             # keys that grow along the sequence: the running maximum moves
+    (1, 65, 2, 1, 63, 0.0), (2, 200, 4, 2, 33, 0.5)])             # pasts that end inside a 64-position step; two sequences, growing keys
 def test_attn_prefill_against_oracle(nnc, oracle_mod, batch, T, nq, nkv, n_past, growth):
     """Causal prompt-phase attention: query s sees cache positions 0 .. n_past + s.  Rows are checked against the
     oracle's single-query attention over the matching cache prefix (sampled rows, all heads of those rows).  With
