@@ -40,6 +40,14 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// Tracing builds: the roles keep per-step time stamps in shared memory (slot [step][what]; row 31 belongs to the CTA as a
+// whole) and thread 0 turns them into records when the CTA is done, so that recording is not on the path it measures.
+#ifdef NNC_TRACE
+#define NNC_TS(j, k, t) do { if (traced && (j) < 32) trace_ts[(j)][(k)] = (t); } while (0)
+#else
+#define NNC_TS(j, k, t) do { } while (0)
+#endif
+
 template <bool OUT_FP16>
 __global__ void __launch_bounds__(kFThreads, 2)
 attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const PfParams p) {
@@ -64,9 +72,6 @@ attn_prefill_f16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     (void)tr_cta;
 #ifdef NNC_TRACE
     __shared__ unsigned long long trace_ts[32][8];
-#define NNC_TS(j, k, t) do { if (traced && (j) < 32) trace_ts[(j)][(k)] = (t); } while (0)
-#else
-#define NNC_TS(j, k, t) do { } while (0)
 #endif
     // The grid is one-dimensional and ordered by decreasing length: all (head, sequence) pairs of the last query tile
     // (the most cache tiles) first, the first query tile last, so that the long CTAs never start late.  Neighbouring

@@ -111,7 +111,7 @@ def test_tracing_build_compiles(tmp_path):
     the product library, so all that is checked here is that the instrumented sources still compile."""
     from paper_2512_21571_b200 import build
     csrc = os.path.join(ROOT, "paper_2512_21571_b200", "csrc")
-    for name in ("decode_misc.cu", "nnc_api.cu"):
+    for name in ("decode_misc.cu", "nnc_api.cu", "attn_prefill_f16.cu"):
         cmd = ["nvcc", *build.NVCC_FLAGS, "-DNNC_TRACE", "-DNNC_TUNING", "-c", os.path.join(csrc, name), "-o",
                str(tmp_path / (name + ".o"))]
         r = subprocess.run(cmd, capture_output=True, text=True)
