@@ -96,7 +96,10 @@ struct SmemLayout {
     static constexpr int kX = (SWAP ? BN : kBM) * kBK * 2;
     static constexpr int kAtom = kW + kX * (SPLIT ? 2 : 1);   // one 64-wide K slab of every operand
     static constexpr int kStage = KA * kAtom;                 // KA slabs per pipeline stage
-    static constexpr int kStagesFit = (192 * 1024) / kStage;
+    // <= 32 tokens: the ring stays under 160 KB (three stages of 48 KB).  Measured on the batch-32 decode step: 11.17 ms
+    // with a 192 KB ring (4 x 48 KB; 7 x 24 KB = 168 KB: 10.8), 10.63 ms with 144 KB, 10.78 ms even with 96 KB (4 x 24 KB)
+    // -- ring depth hardly matters, a CTA that leaves a quarter of the SM's shared memory free does.
+    static constexpr int kStagesFit = ((SWAP && BN == 32 ? 160 : 192) * 1024) / kStage;
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr int kBytes = kStages * kStage + 1024 /*align slack*/ + 256 /*barriers*/;
     static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
@@ -642,9 +645,9 @@ cudaError_t launch_tc_ka(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, c
     return cudaLaunchKernelEx(&cfg, kern, map_w, map_x, map_x_lo, p);
 }
 
-// Few tokens (weights on the M side): a stage carries 2 consecutive K slabs (four stages of 48 KB at <= 32 tokens,
-// three of 64 KB at <= 64), each slab with its own full barrier.  Measured on the batch-32 decode step: 2 slabs per
-// stage 11.25 ms, 4 slabs (two stages of 96 KB) 11.33 ms, 1 slab (eight stages) 11.35 ms.
+// Few tokens (weights on the M side): a stage carries 2 consecutive K slabs (three stages of 48 KB at <= 32 tokens,
+// three of 64 KB at <= 64), each slab with its own full barrier.  Measured on the batch-32 decode step with a 192 KB
+// ring: 2 slabs per stage 11.25 ms, 4 slabs (two stages of 96 KB) 11.33 ms, 1 slab (eight stages) 11.35 ms.
 template <int BN, bool SWAP, int EPI, bool SPLIT>
 cudaError_t launch_tc(const LaunchCtx &lc, const bf16 *X, const bf16 *X_lo, const bf16 *W, void *Y, void *Y_lo, int T, int N,
                       int K, int ldy, int *status, const GemmScratch *scratch) {
