@@ -39,7 +39,12 @@ constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;   // + the producer warp
 constexpr int kMaxStages = 12;
-constexpr int kRingBytes = 192 * 1024;          // more than half an SM: exactly one of these CTAs fits per SM
+constexpr int kRingBytes = 192 * 1024;          // the most a ring may take (geometry: a stage is at most a quarter of it)
+// What a ring actually takes: as many stages as fit in 152 KB (three at the largest stage size).  Measured on the 8B
+// decode step: 192 KB rings 2.887 ms, 168 KB 2.82, 160 KB 2.82, 152 KB 2.809, 144 KB 2.809, two 48 KB stages 2.98 --
+// beyond three stages depth buys nothing, and a CTA that leaves a third of the SM's shared memory to the L1 cache is
+// faster; still more than half an SM, so exactly one of these CTAs fits per SM.
+constexpr int kRingTarget = 152 * 1024;
 constexpr int kBlockRows = 64;                    // rows between two folds of the partial sums
 constexpr uint32_t kSpinLimit = 1u << 22;         // try_wait attempts before a wait gives up (each may block ~us)
 
@@ -532,7 +537,7 @@ cudaError_t launch_gemv_stream(const LaunchCtx &lc, const void *W, const float *
     p.x = x; p.y = y; p.gain = gain; p.eps = eps; p.n_out = n_out; p.K = n_in;
     p.kw = n_in / p.ksplit;
     const int stage_bytes = p.rps * n_in * wb;
-    int S = kRingBytes / stage_bytes;
+    int S = kRingTarget / stage_bytes;
     if (S > kMaxStages) S = kMaxStages;
     if (S < 2) return cudaErrorInvalidValue;
     p.stages = S;
