@@ -42,8 +42,9 @@ constexpr int kMaxStages = 12;
 constexpr int kRingBytes = 192 * 1024;          // the most a ring may take (geometry: a stage is at most a quarter of it)
 // What a ring actually takes: as many stages as fit in 152 KB (three at the largest stage size).  Measured on the 8B
 // decode step: 192 KB rings 2.887 ms, 168 KB 2.82, 160 KB 2.82, 152 KB 2.809, 144 KB 2.809, two 48 KB stages 2.98 --
-// beyond three stages depth buys nothing, and a CTA that leaves a third of the SM's shared memory to the L1 cache is
-// faster; still more than half an SM, so exactly one of these CTAs fits per SM.
+// beyond three stages depth buys nothing, while a CTA under the 164 KB carve-out step leaves 92 instead of 28 KB of L1 to
+// the kernel that follows it on the SM (the flash-decode reads K/V through L1) and room for that kernel's CTAs beside
+// it.  Still more than half an SM, so exactly one of these CTAs fits per SM.
 constexpr int kRingTarget = 152 * 1024;
 constexpr int kBlockRows = 64;                    // rows between two folds of the partial sums
 constexpr uint32_t kSpinLimit = 1u << 22;         // try_wait attempts before a wait gives up (each may block ~us)
