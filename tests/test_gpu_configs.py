@@ -3,7 +3,7 @@ oracle's tokens.  Weights are generated once on the GPU (seeded) and copied to t
 
 Configs 2, 3 and 4 run at their stated lengths (NNC_TEST_STEPS shortens the decode part for quick runs).  Config 5
 is too large for the oracle as a whole (~114 TFLOP of CPU work in mode 1, 32 x 8192 cached positions in mode 2), so
-the oracle's share is: mode 1 -- one full-depth 256-token sequence, plus sequence 0 of the full 4 x 2048 call over
+the oracle's share is: mode 1 -- one full-depth 192-token sequence, plus sequence 0 of the full 4 x 2048 call over
 the first NNC_TEST_LAYERS (default 2) layers at all 2048 positions, plus batch independence at the full size;
 mode 2 -- two of the 32 sequences.  Error statistics are printed and, if NNC_PARITY_STATS names a file, appended.
 """
@@ -152,9 +152,10 @@ def test_config4_qwen3_8b_ctx4096_decode_fp8_weight_format(oracle_mod):
     m.close(); o.close()
 
 
-def test_config5_mode1_qwen3_8b_prefill256_full_depth(oracle_mod):
-    # the 8B shape at full depth on one 256-token sequence: what 36 layers do to the error
-    _run(oracle_mod, "qwen3-8b", 4, prefill=int(os.environ.get("NNC_TEST_PREFILL", "256")), decode=STEPS or 2)
+def test_config5_mode1_qwen3_8b_prefill192_full_depth(oracle_mod):
+    # the 8B shape at full depth on one 192-token sequence (one and a half query tiles, so the prompt-phase operand
+    # path for more than 128 tokens): what 36 layers do to the error.  The oracle needs ~1 s per token here.
+    _run(oracle_mod, "qwen3-8b", 4, prefill=int(os.environ.get("NNC_TEST_PREFILL", "192")), decode=STEPS or 2)
 
 
 def test_config5_mode1_qwen3_8b_4x2048_first_layers_vs_oracle(oracle_mod):
@@ -231,7 +232,7 @@ def test_config5_mode2_qwen3_8b_batch32_ctx8192_sampled(oracle_mod):
 def test_config5_mode1_full_size_batch_independence(oracle_mod):
     """The launch configuration the benchmark times (8B shape, 4 x 2048 tokens): every sequence of the batched call
     must equal the same sequence run alone (logits and appended cache rows), which ties the full-size batched call to
-    the single-sequence path that the oracle checks on a 256-token prefix."""
+    the single-sequence path that the oracle checks on a 192-token prefix."""
     name, seed, B, T = "qwen3-8b", 4, 4, 2048
     shape = synth.SHAPES[name]
     m, o, w = make_pair(oracle_mod, shape, seed, max_seq=T, max_batch=B, max_tokens=B * T)
